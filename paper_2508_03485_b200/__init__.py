@@ -1,0 +1,12 @@
+"""B200 (sm_100a) quantized-linear path of LRQ-DiT: thin Python binding over the C-ABI library.
+
+Every step of the path (rotation, per-token quantization, TLQ decode + tcgen05 contraction,
+epilogue, TLQ weight quantization) runs in the CUDA library ``liblrq_b200.so``; this package only
+marshals arguments.  There is no CPU fallback: importing works without a GPU, calling does not.
+"""
+from .binding import (  # noqa: F401
+    StackPlan,
+    load_library, LrqError, TLQWeights, QLayer,
+    lrq_tlq_quantize_weights, lrq_rotate_quantize_act, lrq_qlinear, lrq_qlinear_stack, lrq_qgemm_codes,
+    lrq_device_status, lrq_version, ROT_NONE, ROT_HADAMARD, ROT_DENSE, ACT_ASYM, ACT_SYM, F32, F16, BF16,
+)

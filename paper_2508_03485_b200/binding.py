@@ -1,0 +1,264 @@
+"""ctypes binding of ``include/lrq.h``.  Argument marshalling only; torch supplies device memory
+and streams.  Function names are those of the C ABI."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIBPATH = os.path.join(_HERE, "liblrq_b200.so")
+
+ROT_NONE, ROT_HADAMARD, ROT_DENSE = 0, 1, 2
+ACT_ASYM, ACT_SYM = 0, 1
+F32, F16, BF16 = 0, 1, 2
+_TORCH_DT = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16}
+
+EXPORTS = [
+    "lrq_tlq_quantize_weights", "lrq_act_workspace_bytes", "lrq_rotate_quantize_act", "lrq_layer_create",
+    "lrq_layer_destroy", "lrq_workspace_bytes", "lrq_qlinear", "lrq_qlinear_stack", "lrq_qgemm_codes",
+    "lrq_device_status", "lrq_status_string", "lrq_version",
+]
+
+
+class LrqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = load_library().lrq_status_string(code).decode()
+        super().__init__(f"{where}: {msg} (status {code})")
+
+
+class _TlqParams(C.Structure):
+    _fields_ = [("w_bits", C.c_int), ("group_size", C.c_int), ("integerize_I", C.c_int),
+                ("n_alpha", C.c_int), ("n_beta", C.c_int),
+                ("alpha", C.POINTER(C.c_double)), ("beta", C.POINTER(C.c_double))]
+
+
+class _ActParams(C.Structure):
+    _fields_ = [("kind", C.c_int), ("had_block", C.c_int), ("R_bf16", C.c_void_p),
+                ("a_bits", C.c_int), ("mode", C.c_int)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Load ``liblrq_b200.so`` (built in-tree by ``paper_2508_03485_b200/build.py``).  Raises if it is
+    missing: there is no other implementation to fall back to."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIBPATH):
+        raise RuntimeError(f"{_LIBPATH} not found: build it with `python -m paper_2508_03485_b200.build` "
+                           "(nvcc, sm_100a); there is no CPU fallback")
+    lib = C.CDLL(_LIBPATH)
+    vp, ci, cl, sz = C.c_void_p, C.c_int, C.c_long, C.c_size_t
+    lib.lrq_tlq_quantize_weights.argtypes = [vp, ci, ci, C.POINTER(_TlqParams), vp, vp, vp, vp, vp, sz, vp]
+    lib.lrq_act_workspace_bytes.argtypes = [ci, ci, C.POINTER(_ActParams)]
+    lib.lrq_act_workspace_bytes.restype = sz
+    lib.lrq_rotate_quantize_act.argtypes = [vp, ci, ci, cl, C.POINTER(_ActParams), vp, vp, vp, vp, sz, vp]
+    lib.lrq_layer_create.argtypes = [C.POINTER(vp), ci, ci, ci, ci, vp, vp, vp, vp, vp, C.POINTER(_ActParams)]
+    lib.lrq_layer_destroy.argtypes = [vp]
+    lib.lrq_layer_destroy.restype = None
+    lib.lrq_workspace_bytes.argtypes = [vp, ci]
+    lib.lrq_workspace_bytes.restype = sz
+    lib.lrq_qlinear.argtypes = [vp, vp, ci, cl, vp, ci, cl, vp, sz, vp]
+    lib.lrq_qlinear_stack.argtypes = [C.POINTER(vp), ci, C.POINTER(vp), C.POINTER(ci), C.POINTER(cl),
+                                      C.POINTER(vp), ci, C.POINTER(cl), vp, sz, vp]
+    lib.lrq_qgemm_codes.argtypes = [vp, vp, vp, vp, ci, vp, ci, cl, ci, vp]
+    lib.lrq_device_status.argtypes = [vp]
+    lib.lrq_status_string.argtypes = [ci]
+    lib.lrq_status_string.restype = C.c_char_p
+    for name in EXPORTS:
+        getattr(lib, name)
+    _lib = lib
+    return lib
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> C.c_void_p:
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise LrqError(code, where)
+
+
+def _need_cuda(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise ValueError("device tensors required (there is no CPU path)")
+
+
+def lrq_version() -> int:
+    return int(load_library().lrq_version())
+
+
+def lrq_device_status(stream=None) -> int:
+    return int(load_library().lrq_device_status(_stream(stream)))
+
+
+# ------------------------------------------------------------------------------------------------
+@dataclass
+class TLQWeights:
+    codes: torch.Tensor    # uint8 [N, K/2]
+    levels: torch.Tensor   # float32 [N, K/G, 2^b]
+    meta: torch.Tensor     # float64 [N, K/G, 6]
+    wsum: torch.Tensor     # float32 [N]
+    w_bits: int
+    group: int             # 0 = per output channel
+
+
+def lrq_tlq_quantize_weights(W_rot: torch.Tensor, w_bits: int, group_size: int = 0, integerize_I: int = 7,
+                             alpha: Sequence[float] = (1.0,), beta: Sequence[float] = (1.0,),
+                             stream=None) -> TLQWeights:
+    """TLQ weight quantization (Sec. 4.1, Eqs. 4-9) of a device float32 [N,K] matrix."""
+    _need_cuda(W_rot)
+    assert W_rot.dtype == torch.float32 and W_rot.is_contiguous() and W_rot.dim() == 2
+    N, K = W_rot.shape
+    G = K if group_size <= 0 else group_size
+    dev = W_rot.device
+    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+    levels = torch.empty((N, max(1, K // max(G, 1)), 1 << w_bits), dtype=torch.float32, device=dev)
+    meta = torch.empty((N, max(1, K // max(G, 1)), 6), dtype=torch.float64, device=dev)
+    wsum = torch.empty((N,), dtype=torch.float32, device=dev)
+    a = (C.c_double * len(alpha))(*[float(v) for v in alpha])
+    b = (C.c_double * len(beta))(*[float(v) for v in beta])
+    p = _TlqParams(int(w_bits), int(group_size), int(integerize_I), len(alpha), len(beta),
+                   C.cast(a, C.POINTER(C.c_double)), C.cast(b, C.POINTER(C.c_double)))
+    rc = load_library().lrq_tlq_quantize_weights(_ptr(W_rot), N, K, C.byref(p), _ptr(codes), _ptr(levels),
+                                                 _ptr(meta), _ptr(wsum), None, 0, _stream(stream))
+    _check(rc, "lrq_tlq_quantize_weights")
+    return TLQWeights(codes, levels, meta, wsum, int(w_bits), int(group_size))
+
+
+def _act_params(kind: int, had_block: int, R: Optional[torch.Tensor], a_bits: int, mode: int) -> _ActParams:
+    return _ActParams(int(kind), int(had_block), 0 if R is None else R.data_ptr(), int(a_bits), int(mode))
+
+
+def lrq_rotate_quantize_act(X: torch.Tensor, kind: int, a_bits: int, had_block: int = 0,
+                            R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM,
+                            workspace: Optional[torch.Tensor] = None, stream=None):
+    """Rotation + per-token quantization (Eq. 12, Eq. 1) of device bf16 [M,K] activations.
+    Returns (codes uint8, scale float32 [M], zero_point int32 [M])."""
+    _need_cuda(X, R, workspace)
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    lib = load_library()
+    p = _act_params(kind, had_block, R, a_bits, mode)
+    need = int(lib.lrq_act_workspace_bytes(M, K, C.byref(p)))
+    if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
+        workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
+    dev = X.device
+    codes = torch.empty((M, K * a_bits // 8), dtype=torch.uint8, device=dev)
+    scale = torch.empty((M,), dtype=torch.float32, device=dev)
+    zp = torch.empty((M,), dtype=torch.int32, device=dev)
+    wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.lrq_rotate_quantize_act(_ptr(X), M, K, X.stride(0), C.byref(p), _ptr(codes), _ptr(scale), _ptr(zp),
+                                     _ptr(workspace), wsb, _stream(stream))
+    _check(rc, "lrq_rotate_quantize_act")
+    return codes, scale, zp
+
+
+class QLayer:
+    """Owner of one ``lrq_layer`` handle and of the device tensors it points to."""
+
+    def __init__(self, tlq: TLQWeights, N: int, K: int, kind: int, a_bits: int, had_block: int = 0,
+                 R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM,
+                 wscale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None):
+        _need_cuda(tlq.codes, tlq.levels, tlq.wsum, R, wscale, bias)
+        self.tlq, self.N, self.K, self.R, self.wscale, self.bias = tlq, N, K, R, wscale, bias
+        self.kind, self.a_bits, self.had_block, self.mode = kind, a_bits, had_block, mode
+        self._p = _act_params(kind, had_block, R, a_bits, mode)
+        h = C.c_void_p()
+        rc = load_library().lrq_layer_create(C.byref(h), N, K, tlq.w_bits, tlq.group, _ptr(tlq.codes),
+                                             _ptr(tlq.levels), _ptr(tlq.wsum), _ptr(wscale), _ptr(bias),
+                                             C.byref(self._p))
+        _check(rc, "lrq_layer_create")
+        self.handle = h
+
+    def workspace_bytes(self, M: int) -> int:
+        return int(load_library().lrq_workspace_bytes(self.handle, int(M)))
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load_library().lrq_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _ws(workspace: Optional[torch.Tensor], need: int, device) -> torch.Tensor:
+    if workspace is None or workspace.numel() * workspace.element_size() < need:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+    return workspace
+
+
+def lrq_qlinear(layer: QLayer, X: torch.Tensor, y_dtype: int = F32, out: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Y = quantized-linear(X) for device bf16 X [M,K] (Eq. 12 -> Eq. 1 -> Eq. 10 -> scaling)."""
+    _need_cuda(X, out, workspace)
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1 and X.shape[1] == layer.K
+    M = X.shape[0]
+    if out is None:
+        out = torch.empty((M, layer.N), dtype=_TORCH_DT[y_dtype], device=X.device)
+    assert out.dtype == _TORCH_DT[y_dtype] and out.stride(1) == 1
+    workspace = _ws(workspace, layer.workspace_bytes(M), X.device)
+    rc = load_library().lrq_qlinear(layer.handle, _ptr(X), M, X.stride(0), _ptr(out), y_dtype, out.stride(0),
+                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(rc, "lrq_qlinear")
+    return out
+
+
+class StackPlan:
+    """Host-side argument arrays of one lrq_qlinear_stack call, built once and reused."""
+
+    def __init__(self, layers: List[QLayer], Xs: List[torch.Tensor], Ys: List[torch.Tensor], y_dtype: int):
+        n = len(layers)
+        vp = C.c_void_p
+        self.n, self.y_dtype = n, y_dtype
+        self.layers = (vp * n)(*[l.handle for l in layers])
+        self.X = (vp * n)(*[x.data_ptr() for x in Xs])
+        self.Y = (vp * n)(*[y.data_ptr() for y in Ys])
+        self.M = (C.c_int * n)(*[x.shape[0] for x in Xs])
+        self.ldx = (C.c_long * n)(*[x.stride(0) for x in Xs])
+        self.ldy = (C.c_long * n)(*[y.stride(0) for y in Ys])
+        self.need = max(l.workspace_bytes(x.shape[0]) for l, x in zip(layers, Xs))
+        self._keep = (layers, Xs, Ys)
+
+
+def lrq_qlinear_stack(plan: StackPlan, workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    """All layers of ``plan`` back to back on one stream, one shared workspace."""
+    dev = plan._keep[1][0].device
+    workspace = _ws(workspace, plan.need, dev)
+    rc = load_library().lrq_qlinear_stack(plan.layers, plan.n, plan.X, plan.M, plan.ldx, plan.Y, plan.y_dtype,
+                                          plan.ldy, _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                          _stream(stream))
+    _check(rc, "lrq_qlinear_stack")
+
+
+def lrq_qgemm_codes(layer: QLayer, a_codes: torch.Tensor, a_scale: torch.Tensor, a_zp: torch.Tensor,
+                    y_dtype: int = F32, impl: int = 0, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Contraction + epilogue alone (Eq. 10) on codes from lrq_rotate_quantize_act.
+    impl 0: tcgen05 kernel, 1: CUDA-core baseline kernel."""
+    _need_cuda(a_codes, a_scale, a_zp, out)
+    M = a_codes.shape[0]
+    if out is None:
+        out = torch.empty((M, layer.N), dtype=_TORCH_DT[y_dtype], device=a_codes.device)
+    rc = load_library().lrq_qgemm_codes(layer.handle, _ptr(a_codes), _ptr(a_scale), _ptr(a_zp), M, _ptr(out),
+                                        y_dtype, out.stride(0), impl, _stream(stream))
+    _check(rc, "lrq_qgemm_codes")
+    return out

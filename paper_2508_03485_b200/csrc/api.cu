@@ -1,0 +1,195 @@
+// C-ABI entry points: argument checks, workspace carving, launches.  No entry point allocates
+// device memory or synchronises (lrq_device_status excepted, which reads one word back).
+#include "lrq_internal.cuh"
+#include <new>
+
+// Status word written by a kernel whose bounded wait expired.  A file-scope device variable: in
+// host code its name is only a handle, the device address comes from cudaGetSymbolAddress (for
+// the device that is current at the time of the call).
+__device__ int g_lrq_status_word;
+
+int* lrq_status_word() {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_lrq_status_word) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    return p;
+}
+
+static lrq_status check_act(const lrq_act_params* p, int K) {
+    if (!p) return LRQ_ERR_INVALID_ARG;
+    if (p->a_bits != 4 && p->a_bits != 8) return LRQ_ERR_UNSUPPORTED;
+    if (p->mode != LRQ_ACT_ASYM && p->mode != LRQ_ACT_SYM) return LRQ_ERR_INVALID_ARG;
+    if (K <= 0 || K % 8) return LRQ_ERR_UNSUPPORTED;
+    switch (p->kind) {
+        case LRQ_ROT_NONE: break;
+        case LRQ_ROT_HADAMARD:
+            if (!lrq_is_pow2(p->had_block) || p->had_block < 8 || p->had_block > 4096 || K % p->had_block)
+                return LRQ_ERR_UNSUPPORTED;
+            break;
+        case LRQ_ROT_DENSE:
+            if (!p->R_bf16) return LRQ_ERR_INVALID_ARG;
+            if (!lrq_aligned(p->R_bf16, 16)) return LRQ_ERR_INVALID_ARG;
+            break;
+        default: return LRQ_ERR_INVALID_ARG;
+    }
+    return LRQ_OK;
+}
+
+extern "C" size_t lrq_act_workspace_bytes(int M, int K, const lrq_act_params* p) {
+    if (!p || M <= 0 || K <= 0) return 0;
+    return p->kind == LRQ_ROT_DENSE ? lrq_round_up((size_t)M * K * sizeof(float), 256) : 0;
+}
+
+extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long ldx, const lrq_act_params* p,
+                                              uint8_t* a_codes, float* a_scale, int32_t* a_zp,
+                                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!X || !a_codes || !a_scale || !a_zp || M <= 0) return LRQ_ERR_INVALID_ARG;
+    lrq_status st = check_act(p, K);
+    if (st != LRQ_OK) return st;
+    if (ldx < K || (ldx % 8) || !lrq_aligned(X, 16) || !lrq_aligned(a_codes, 16)) return LRQ_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (p->kind == LRQ_ROT_DENSE) {
+        const size_t need = lrq_act_workspace_bytes(M, K, p);
+        if (!workspace || workspace_bytes < need || !lrq_aligned(workspace, 256)) return LRQ_ERR_WORKSPACE;
+        float* Yr = static_cast<float*>(workspace);
+        st = lrq_launch_rotgemm(X, M, K, ldx, p->R_bf16, Yr, stream);
+        if (st != LRQ_OK) return st;
+        return lrq_launch_quantize_f32(Yr, M, K, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
+    }
+    const int B = p->kind == LRQ_ROT_HADAMARD ? p->had_block : 1;
+    return lrq_launch_rotq_hadamard(X, M, K, ldx, B, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
+}
+
+extern "C" lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size,
+                                       const uint8_t* codes, const float* levels, const float* wsum,
+                                       const float* wscale, const float* bias, const lrq_act_params* act) {
+    if (!out) return LRQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!codes || !levels || !wsum || N <= 0 || K <= 0) return LRQ_ERR_INVALID_ARG;
+    if (w_bits < 2 || w_bits > 4) return LRQ_ERR_UNSUPPORTED;
+    const int G = group_size > 0 ? group_size : K;
+    if (K % G || G % 8) return LRQ_ERR_UNSUPPORTED;
+    lrq_status st = check_act(act, K);
+    if (st != LRQ_OK) return st;
+    if (!lrq_aligned(codes, 16) || !lrq_aligned(levels, 16)) return LRQ_ERR_INVALID_ARG;
+    lrq_layer* L = new (std::nothrow) lrq_layer;
+    if (!L) return LRQ_ERR_INVALID_ARG;
+    L->N = N; L->K = K; L->w_bits = w_bits; L->group = G;
+    L->codes = codes; L->levels = levels; L->wsum = wsum; L->wscale = wscale; L->bias = bias;
+    L->act = *act;
+    *out = L;
+    return LRQ_OK;
+}
+
+extern "C" void lrq_layer_destroy(lrq_layer* L) { delete L; }
+
+namespace {
+struct WsLayout { size_t codes, scale, zp, rot, total; };
+WsLayout ws_layout(const lrq_layer* L, int M) {
+    WsLayout w;
+    size_t off = 0;
+    w.codes = off; off += lrq_round_up((size_t)M * L->K * L->act.a_bits / 8, 256);
+    w.scale = off; off += lrq_round_up((size_t)M * sizeof(float), 256);
+    w.zp = off;    off += lrq_round_up((size_t)M * sizeof(int32_t), 256);
+    w.rot = off;   off += lrq_act_workspace_bytes(M, L->K, &L->act);
+    w.total = off;
+    return w;
+}
+}  // namespace
+
+extern "C" size_t lrq_workspace_bytes(const lrq_layer* L, int M) {
+    if (!L || M <= 0) return 0;
+    return ws_layout(L, M).total;
+}
+
+static lrq_status check_out(const void* Y, lrq_dtype dt, long ldy, int N) {
+    if (!Y || ldy < N) return LRQ_ERR_INVALID_ARG;
+    if (dt != LRQ_F32 && dt != LRQ_F16 && dt != LRQ_BF16) return LRQ_ERR_INVALID_ARG;
+    const size_t es = dt == LRQ_F32 ? 4 : 2;
+    if (!lrq_aligned(Y, 16) || ((size_t)ldy * es) % 16) return LRQ_ERR_INVALID_ARG;
+    return LRQ_OK;
+}
+
+static lrq_status qgemm_dispatch(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
+                                 const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, int impl,
+                                 cudaStream_t st) {
+    if (impl == 1) return lrq_launch_qgemm_simple(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, st);
+    lrq_status s = lrq_launch_qgemm_tc(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, st);
+    if (s == LRQ_ERR_UNSUPPORTED && impl < 0)       // automatic choice: shapes outside the tensor-core kernel
+        return lrq_launch_qgemm_simple(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, st);
+    return s;
+}
+
+extern "C" lrq_status lrq_qgemm_codes(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
+                                      const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, int impl,
+                                      void* cuda_stream) {
+    if (!L || !a_codes || !a_scale || !a_zp || M <= 0) return LRQ_ERR_INVALID_ARG;
+    if (impl != 0 && impl != 1) return LRQ_ERR_INVALID_ARG;
+    lrq_status st = check_out(Y, dt, ldy, L->N);
+    if (st != LRQ_OK) return st;
+    if (!lrq_aligned(a_codes, 16)) return LRQ_ERR_INVALID_ARG;
+    return qgemm_dispatch(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, impl, (cudaStream_t)cuda_stream);
+}
+
+extern "C" lrq_status lrq_qlinear(const lrq_layer* L, const void* X, int M, long ldx, void* Y, lrq_dtype dt, long ldy,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!L || !X || M <= 0) return LRQ_ERR_INVALID_ARG;
+    lrq_status st = check_out(Y, dt, ldy, L->N);
+    if (st != LRQ_OK) return st;
+    const WsLayout w = ws_layout(L, M);
+    if (!workspace || workspace_bytes < w.total || !lrq_aligned(workspace, 256)) return LRQ_ERR_WORKSPACE;
+    char* base = static_cast<char*>(workspace);
+    uint8_t* a_codes = reinterpret_cast<uint8_t*>(base + w.codes);
+    float* a_scale = reinterpret_cast<float*>(base + w.scale);
+    int32_t* a_zp = reinterpret_cast<int32_t*>(base + w.zp);
+    st = lrq_rotate_quantize_act(X, M, L->K, ldx, &L->act, a_codes, a_scale, a_zp, base + w.rot,
+                                 w.total - w.rot, cuda_stream);
+    if (st != LRQ_OK) return st;
+    return qgemm_dispatch(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, -1, (cudaStream_t)cuda_stream);
+}
+
+extern "C" lrq_status lrq_qlinear_stack(const lrq_layer* const* layers, int n_layers, const void* const* X,
+                                        const int* M, const long* ldx, void* const* Y, lrq_dtype dt,
+                                        const long* ldy, void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream) {
+    if (!layers || !X || !M || !ldx || !Y || !ldy || n_layers <= 0) return LRQ_ERR_INVALID_ARG;
+    // validate everything before the first launch
+    for (int i = 0; i < n_layers; ++i) {
+        if (!layers[i] || !X[i] || M[i] <= 0) return LRQ_ERR_INVALID_ARG;
+        lrq_status st = check_out(Y[i], dt, ldy[i], layers[i]->N);
+        if (st != LRQ_OK) return st;
+        if (!workspace || workspace_bytes < lrq_workspace_bytes(layers[i], M[i])) return LRQ_ERR_WORKSPACE;
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        lrq_status st = lrq_qlinear(layers[i], X[i], M[i], ldx[i], Y[i], dt, ldy[i], workspace, workspace_bytes,
+                                    cuda_stream);
+        if (st != LRQ_OK) return st;
+    }
+    return LRQ_OK;
+}
+
+extern "C" int lrq_device_status(void* cuda_stream) {
+    int* w = lrq_status_word();
+    if (!w) return -1;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, w, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)cuda_stream) != cudaSuccess) return -1;
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return -1;
+    if (v) cudaMemsetAsync(w, 0, sizeof(int), (cudaStream_t)cuda_stream);
+    return v;
+}
+
+extern "C" const char* lrq_status_string(lrq_status s) {
+    switch (s) {
+        case LRQ_OK: return "ok";
+        case LRQ_ERR_INVALID_ARG: return "invalid argument";
+        case LRQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case LRQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case LRQ_ERR_CUDA: return "CUDA call failed";
+        case LRQ_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown";
+}
+
+extern "C" int lrq_version(void) { return 100; }

@@ -1,0 +1,43 @@
+// Internal declarations shared by the translation units of the CUDA library.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include "../../include/lrq.h"
+
+#define LRQ_CUDA_TRY(expr)                                   \
+    do {                                                     \
+        cudaError_t e__ = (expr);                            \
+        if (e__ != cudaSuccess) { (void)cudaGetLastError(); return LRQ_ERR_CUDA; } \
+    } while (0)
+
+static inline bool lrq_is_pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+static inline bool lrq_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+static inline size_t lrq_round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct lrq_layer {
+    int N, K, w_bits, group;          // group == K for per-channel tables
+    const uint8_t* codes;
+    const float* levels;
+    const float* wsum;
+    const float* wscale;
+    const float* bias;
+    lrq_act_params act;
+};
+
+// Device status word: written by a kernel whose bounded wait expired.
+int* lrq_status_word();               // device address of the word (allocated lazily, once per process)
+
+// rotq.cu
+lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B, int a_bits, int mode,
+                                    uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
+lrq_status lrq_launch_quantize_f32(const float* Y, int M, int K, long ldy, int a_bits, int mode,
+                                   uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
+// rotgemm.cu : Y[M,K] (fp32) = X[M,K] (bf16) . R[K,K] (bf16)
+lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y, cudaStream_t st);
+// qgemm_simple.cu / qgemm_tc.cu
+lrq_status lrq_launch_qgemm_simple(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
+                                   const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);
+lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
+                               const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);

@@ -1,0 +1,97 @@
+// Quantized contraction and epilogue on the CUDA cores (Sec. 4.1, Eq. 10 evaluated exactly).
+//
+// In-library ablation baseline and the path for shapes the tensor-core kernel does not take.
+// A 64x64 output tile per CTA; activation codes and TLQ codes are decoded to fp32 in shared
+// memory (codes through the group's level table), every product q*level is exact in fp32 and
+// the sum is accumulated in fp32.
+#include "lrq_internal.cuh"
+
+namespace {
+
+constexpr int TM = 64, TN = 64, TK = 32;
+
+template <typename OutT> __device__ __forceinline__ OutT cast_out(float v);
+template <> __device__ __forceinline__ float cast_out<float>(float v) { return v; }
+template <> __device__ __forceinline__ __half cast_out<__half>(float v) { return __float2half_rn(v); }
+template <> __device__ __forceinline__ __nv_bfloat16 cast_out<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+qgemm_simple_kernel(const uint8_t* __restrict__ a_codes, const float* __restrict__ a_scale,
+                    const int32_t* __restrict__ a_zp, int M, int N, int K, int a_bits, int w_bits, int G,
+                    const uint8_t* __restrict__ w_codes, const float* __restrict__ levels,
+                    const float* __restrict__ wsum, const float* __restrict__ wscale,
+                    const float* __restrict__ bias, OutT* __restrict__ Y, long ldy) {
+    __shared__ float As[TK][TM + 1];
+    __shared__ float Ws[TK][TN + 1];
+    const int tid = threadIdx.x;
+    const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+    const int tx = tid & 15, ty = tid >> 4;              // 16 x 16 threads, 4 x 4 outputs each
+    const int nlev = 1 << w_bits, ngrp = K / G;
+    float acc[4][4] = {};
+
+    for (int k0 = 0; k0 < K; k0 += TK) {
+        for (int e = tid; e < TM * TK; e += 256) {
+            const int r = e / TK, kk = e % TK, m = m0 + r, k = k0 + kk;
+            float v = 0.f;
+            if (m < M && k < K) {
+                if (a_bits == 8) v = (float)a_codes[(size_t)m * K + k];
+                else v = (float)((a_codes[((size_t)m * K + k) >> 1] >> (4 * (k & 1))) & 0xF);
+            }
+            As[kk][r] = v;
+        }
+        for (int e = tid; e < TN * TK; e += 256) {
+            const int r = e / TK, kk = e % TK, n = n0 + r, k = k0 + kk;
+            float v = 0.f;
+            if (n < N && k < K) {
+                const int u = (w_codes[((size_t)n * K + k) >> 1] >> (4 * (k & 1))) & 0xF;
+                v = levels[((size_t)n * ngrp + k / G) * nlev + u];
+            }
+            Ws[kk][r] = v;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int kk = 0; kk < TK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Ws[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+        const float s = a_scale[m], z = (float)a_zp[m];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n >= N) continue;
+            float y = s * fmaf(z, wsum[n], acc[i][j]);
+            if (wscale) y *= wscale[n];
+            if (bias) y += bias[n];
+            Y[(size_t)m * ldy + n] = cast_out<OutT>(y);
+        }
+    }
+}
+
+}  // namespace
+
+lrq_status lrq_launch_qgemm_simple(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
+                                   const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st) {
+    dim3 grid((L->N + TN - 1) / TN, (M + TM - 1) / TM), block(256);
+#define LRQ_GO(T)                                                                                              \
+    qgemm_simple_kernel<T><<<grid, block, 0, st>>>(a_codes, a_scale, a_zp, M, L->N, L->K, L->act.a_bits,       \
+                                                   L->w_bits, L->group, L->codes, L->levels, L->wsum,          \
+                                                   L->wscale, L->bias, static_cast<T*>(Y), ldy)
+    if (dt == LRQ_F32) LRQ_GO(float);
+    else if (dt == LRQ_F16) LRQ_GO(__half);
+    else LRQ_GO(__nv_bfloat16);
+#undef LRQ_GO
+    LRQ_CUDA_TRY(cudaGetLastError());
+    return LRQ_OK;
+}

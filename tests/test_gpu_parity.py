@@ -1,0 +1,178 @@
+"""GPU parity: every step of the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs.  Small shapes are compared element by element (several tiles plus a ragged tail); the
+BASELINE-sized layers are run in full on the GPU and compared on sampled token rows, which the oracle
+computes one by one (tokens are independent)."""
+import numpy as np
+import pytest
+import torch
+
+import parity as PU
+from lrq_workloads import (LayerSpec, bf16_bits_to_f64, config_layers, default_clip_grid, f32_to_bf16_bits,
+                           make_activations, make_orthogonal, make_weights)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2508_03485_b200 as P
+    P.load_library()
+    return P
+
+
+# --------------------------------------------------------------------------------------------- rotq
+@pytest.mark.parametrize("M,K,B,a_bits,mode", [
+    (1, 128, 128, 8, 0), (7, 1152, 128, 8, 0), (129, 1024, 1024, 4, 0), (33, 1536, 512, 4, 0),
+    (5, 6144, 2048, 4, 0), (3, 12288, 4096, 4, 0), (17, 3072, 1024, 4, 1), (64, 4608, 128, 8, 1),
+    (9, 64, 8, 8, 0), (12, 256, 16, 4, 0), (300, 1152, 128, 4, 0), (2, 512, 64, 8, 0),
+])
+def test_rotate_quantize_hadamard(P, orc, M, K, B, a_bits, mode):
+    xb = make_activations(100 + M + K, M, K)
+    q, s, z = P.lrq_rotate_quantize_act(PU.bf16_to_device(xb), P.ROT_HADAMARD, a_bits, B, mode=mode)
+    Yr = orc.rotate_hadamard_fwht(bf16_bits_to_f64(xb), B)
+    oq, os_, oz = orc.quantize_act(Yr, a_bits, mode)
+    PU.check_act(PU.act_codes_to_numpy(q, a_bits), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, f"rotq {M}x{K} B{B}")
+
+
+def test_rotate_quantize_edge_tokens(P, orc):
+    # constant token, all-zero token, a single spike (Lemma 1), values at the bf16 extremes of the workload
+    K, B = 256, 128
+    x = np.zeros((5, K), dtype=np.float32)
+    x[0] = 2.0
+    x[2, 37] = 245.0
+    x[3] = np.linspace(-300, 300, K)
+    x[4, ::2] = 1.0
+    xb = f32_to_bf16_bits(x)
+    for a_bits in (4, 8):
+        q, s, z = P.lrq_rotate_quantize_act(PU.bf16_to_device(xb), P.ROT_HADAMARD, a_bits, B)
+        oq, os_, oz = orc.quantize_act(orc.rotate_hadamard_fwht(bf16_bits_to_f64(xb), B), a_bits)
+        PU.check_act(PU.act_codes_to_numpy(q, a_bits), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, "edge")
+        assert s[1].item() == 1.0 and z[1].item() == 0          # empty range: unit step
+
+
+def test_rotate_quantize_strided_rows_and_no_rotation(P, orc):
+    M, K = 20, 384
+    xb = make_activations(5, M, 512)
+    xd = PU.bf16_to_device(xb)[:, :K]                          # ldx = 512 > K
+    q, s, z = P.lrq_rotate_quantize_act(xd, P.ROT_NONE, 8)
+    oq, os_, oz = orc.quantize_act(bf16_bits_to_f64(xb[:, :K]), 8)
+    PU.check_act(PU.act_codes_to_numpy(q, 8), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, "none")
+    q, s, z = P.lrq_rotate_quantize_act(xd, P.ROT_HADAMARD, 4, 128)
+    oq, os_, oz = orc.quantize_act(orc.rotate_hadamard_fwht(bf16_bits_to_f64(xb[:, :K]), 128), 4)
+    PU.check_act(PU.act_codes_to_numpy(q, 4), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, "strided")
+
+
+@pytest.mark.parametrize("M,K,a_bits", [(70, 192, 4), (130, 1152, 8), (33, 1536, 4)])
+def test_rotate_quantize_dense(P, orc, M, K, a_bits):
+    xb = make_activations(7, M, K, n_salient=16, salient_x=100.0)
+    Rb = f32_to_bf16_bits(make_orthogonal(3, K).astype(np.float32))
+    q, s, z = P.lrq_rotate_quantize_act(PU.bf16_to_device(xb), P.ROT_DENSE, a_bits, R=PU.bf16_to_device(Rb))
+    oq, os_, oz = orc.quantize_act(orc.rotate_dense(bf16_bits_to_f64(xb), bf16_bits_to_f64(Rb)), a_bits)
+    PU.check_act(PU.act_codes_to_numpy(q, a_bits), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, "dense")
+
+
+# --------------------------------------------------------------------------------------------- tlqw
+@pytest.mark.parametrize("N,K,bits,G", [(16, 128, 3, 0), (33, 1152, 4, 0), (8, 1536, 3, 128), (5, 4608, 4, 0),
+                                        (3, 12288, 4, 0), (64, 256, 2, 64), (7, 64, 4, 8)])
+def test_tlq_quantize_weights(P, orc, N, K, bits, G):
+    W = make_weights(200 + N + K, N, K)
+    W[0, :3] = 0.0
+    g = default_clip_grid()
+    tl = P.lrq_tlq_quantize_weights(torch.from_numpy(W).cuda(), bits, G, 7, g, g)
+    PU.check_tlq(orc, W, tl, bits, G, what=f"tlq {N}x{K} b{bits} G{G}")
+
+
+def test_tlq_degenerate_rows(P, orc):
+    W = np.zeros((4, 64), dtype=np.float32)
+    W[1] = 0.25
+    W[2, ::2], W[2, 1::2] = 0.5, -0.125
+    W[3] = -np.abs(make_weights(1, 1, 64)[0])
+    tl = P.lrq_tlq_quantize_weights(torch.from_numpy(W).cuda(), 3, 0, 7, [1.0, 1.2], [1.0, 1.2])
+    T = orc.tlq_quantize(W.astype(np.float64), 3, 0, 7, [1.0, 1.2], [1.0, 1.2])
+    assert np.array_equal(PU.unpack4(tl.codes.cpu().numpy()).astype(np.int32) - 4, T.codes.astype(np.int32))
+    assert np.array_equal(tl.levels.cpu().numpy().astype(np.float64), T.levels)
+
+
+# --------------------------------------------------------------------------------------------- qgemm
+def _small_layer(P, orc, M, K, N, w_bits, a_bits, G, B, seed, rot="hadamard"):
+    spec = LayerSpec("t", seed, M, K, N, w_bits, a_bits, G, rot, B)
+    W, xb = spec.weights(), spec.activations()
+    layer, tl = PU.gpu_layer(spec, W, P)
+    T = PU.check_tlq(orc, W, tl, w_bits, G, what="small layer")
+    return spec, W, xb, layer, tl, T
+
+
+@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("M,K,N,w_bits,a_bits,G,B", [
+    (70, 256, 72, 4, 8, 0, 128), (129, 1152, 200, 4, 8, 0, 128), (33, 512, 136, 3, 4, 128, 512),
+    (256, 1024, 1024, 3, 4, 0, 1024), (5, 128, 8, 4, 4, 64, 64),
+])
+def test_qgemm_from_oracle_codes(P, orc, impl, M, K, N, w_bits, a_bits, G, B):
+    # the contraction alone: the GPU gets the oracle's activation codes, so only Eq. 10 is compared
+    spec, W, xb, layer, tl, T = _small_layer(P, orc, M, K, N, w_bits, a_bits, G, B, 31)
+    Yo, oq, os_, oz = PU.oracle_layer_rows(orc, spec, xb, T)
+    if a_bits == 8:
+        qd = torch.from_numpy(oq.astype(np.uint8)).cuda()
+    else:
+        qd = torch.from_numpy((oq[:, 0::2] | (oq[:, 1::2] << 4)).astype(np.uint8)).cuda()
+    sd = torch.from_numpy(os_.astype(np.float32)).cuda()
+    zd = torch.from_numpy(oz.astype(np.int32)).cuda()
+    try:
+        Y = P.lrq_qgemm_codes(layer, qd, sd, zd, P.F32, impl)
+    except P.LrqError as e:
+        if impl == 0 and e.code == 2:
+            pytest.skip("shape not taken by the tensor-core kernel")
+        raise
+    assert P.lrq_device_status() == 0
+    PU.check_out(Y.cpu().numpy(), Yo, f"qgemm impl{impl}", rel=2e-6, mx=2e-5)
+
+
+@pytest.mark.parametrize("M,K,N,w_bits,a_bits,G,B,rot", [
+    (70, 256, 72, 4, 8, 0, 128, "hadamard"), (300, 1152, 392, 4, 8, 0, 128, "hadamard"),
+    (129, 1536, 264, 3, 4, 128, 512, "hadamard"), (65, 384, 136, 3, 4, 128, 0, "dense"),
+])
+def test_qlinear_small(P, orc, M, K, N, w_bits, a_bits, G, B, rot):
+    spec, W, xb, layer, tl, T = _small_layer(P, orc, M, K, N, w_bits, a_bits, G, B, 41, rot)
+    Rb = spec.rotation_bf16()
+    Yo, *_ = PU.oracle_layer_rows(orc, spec, xb, T, Rb)
+    X = PU.bf16_to_device(xb)
+    Y = P.lrq_qlinear(layer, X, P.F32)
+    PU.check_out(Y.cpu().numpy(), Yo, "qlinear f32")
+    Yh = P.lrq_qlinear(layer, X, P.F16)
+    PU.check_out(Yh.float().cpu().numpy(), Yo, "qlinear f16", rel=1e-3, mx=1e-2)
+    Yb = P.lrq_qlinear(layer, X, P.BF16).float().cpu().numpy()
+    # bf16 output: within one bf16 ulp (2^-8 relative) of the oracle's value
+    assert (np.abs(Yb - Yo) <= np.abs(Yo) * 2.0 ** -7 + 1e-2 * np.sqrt(np.mean(Yo ** 2)) * 1e-2).all()
+    assert P.lrq_device_status() == 0
+
+
+def test_qlinear_scale_and_bias(P, orc):
+    spec, W, xb, layer, tl, T = _small_layer(P, orc, 40, 256, 96, 4, 8, 0, 128, 43)
+    rng = np.random.default_rng(0)
+    ws, bs = rng.uniform(0.5, 2, 96).astype(np.float32), rng.standard_normal(96).astype(np.float32)
+    layer2 = P.QLayer(tl, 96, 256, P.ROT_HADAMARD, 8, 128, wscale=torch.from_numpy(ws).cuda(),
+                      bias=torch.from_numpy(bs).cuda())
+    X = bf16_bits_to_f64(xb)
+    Yo, *_ = orc.qlinear(X, T, 8, "hadamard", 128, wscale=ws.astype(np.float64), bias=bs.astype(np.float64))
+    Y = P.lrq_qlinear(layer2, PU.bf16_to_device(xb), P.F32)
+    PU.check_out(Y.cpu().numpy(), Yo, "scale+bias")
+
+
+def test_qlinear_stack_matches_single_calls(P):
+    specs = [LayerSpec("a", 51, 64, 256, 72, 4, 8, 0, "hadamard", 128),
+             LayerSpec("b", 52, 48, 512, 40, 3, 4, 128, "hadamard", 512),
+             LayerSpec("c", 53, 33, 128, 136, 4, 8, 0, "dense", 0)]
+    layers, Xs, Ys, refs = [], [], [], []
+    for sp in specs:
+        layer, _ = PU.gpu_layer(sp, sp.weights(), P)
+        X = PU.bf16_to_device(sp.activations())
+        layers.append(layer); Xs.append(X)
+        refs.append(P.lrq_qlinear(layer, X, P.F32))
+        Ys.append(torch.zeros_like(refs[-1]))
+    plan = P.StackPlan(layers, Xs, Ys, P.F32)
+    P.lrq_qlinear_stack(plan)
+    torch.cuda.synchronize()
+    for y, r in zip(Ys, refs):
+        assert torch.equal(y, r)
