@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Throughput of the quantized-linear hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config 1]
+
+One *step* = one pass of the whole online path (rotation -> per-token quantization -> TLQ-decoding
+tensor-core contraction -> epilogue) over every linear of the workload, through `lrq_qlinear_stack`.
+The default workload is the PixArt-shaped W4A8 block (M = 4096 tokens, four linears), inputs already in
+HBM; an L2 flush (a 512 MiB fill) runs between timed steps, outside the timed events.  `value` is the
+whole-job TFLOP/s (2*M*N*K per linear, summed over ranks); `e2e` repeats the measurement with the
+activations in pinned host memory and the outputs read back, copies inside the timed region.
+
+With --gpus N > 1 (under torchrun) every rank runs the same batch on its own GPU: tokens are independent,
+the path has no exchange step, so ranks share nothing but the timing barrier ("weak" scaling).
+
+--impl reference times the fp64 CPU oracle on the host cores on a bounded token sample of the same
+workload and prints the same line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from lrq_workloads import bf16_bits_to_f64, config_layers, default_clip_grid  # noqa: E402
+
+METRIC = "qlinear_tflops"
+UNIT = "TFLOP/s"
+ORACLE_SAMPLE_TOKENS = 128
+
+
+def workload_name(cfg: int) -> str:
+    return {0: "cfg0 single linear W3A4 M=256 K=N=1024",
+            1: "cfg1 PixArt-shape block linears W4A8 M=4096 hidden=1152 (qkv, proj, fc1, fc2)",
+            2: "cfg2 MMDiT-shape linears W3A4 M=4429 hidden=1536 G=128",
+            3: "cfg3 FLUX-shape linears W4A4 M=4608 hidden=3072",
+            4: "cfg4 video-DiT stack 28 blocks W4A8 M=32768 hidden=1152"}[cfg]
+
+
+def layer_flops(specs, M=None):
+    return sum(2.0 * (s.M if M is None else M) * s.N * s.K for s in specs)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+def oracle_step(orc, prepared):
+    """One bounded-sample pass of the oracle over every layer; returns seconds."""
+    t0 = time.perf_counter()
+    for spec, T, X, R in prepared:
+        orc.qlinear(X, T, spec.a_bits, spec.rot, spec.had_block, R)
+    return time.perf_counter() - t0
+
+
+def prepare_oracle(orc, specs, n_tok):
+    g = default_clip_grid()
+    out = []
+    for s in specs:
+        T = orc.tlq_quantize(s.weights().astype(np.float64), s.w_bits, s.group, 7, g, g)
+        X = bf16_bits_to_f64(s.activations(n_tok))
+        Rb = s.rotation_bf16()
+        out.append((s, T, X, None if Rb is None else bf16_bits_to_f64(Rb)))
+    return out
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle as orc
+    orc.build()
+    specs = config_layers(args.config)
+    if args.config == 4:
+        specs = specs[:4]          # one block of the stack is a bounded sample of 28 identical blocks
+    n_tok = ORACLE_SAMPLE_TOKENS
+    prepared = prepare_oracle(orc, specs, n_tok)
+    for _ in range(max(1, min(args.warmup, 2))):
+        oracle_step(orc, prepared)
+    ts = [oracle_step(orc, prepared) for _ in range(args.steps)]
+    sec = float(np.mean(ts))
+    fl = layer_flops(specs, n_tok)
+    val = fl / sec / 1e12
+    sample = f"{n_tok} tokens of each linear (full K, N); work is linear in tokens"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(args.config), "sample": sample},
+            "tokens_per_s": n_tok / sec,
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2508_03485_b200 as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    P.load_library()
+
+    specs = config_layers(args.config)
+    grid = default_clip_grid()
+
+    def bf16_dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+
+    # ---- offline: weights -> TLQ (timed separately), layer handles
+    layers, Xs_host, Xs, Ys = [], [], [], []
+    x_cache = {}
+    tlq_ms, n_weights = 0.0, 0
+    for s in specs:
+        Wd = torch.from_numpy(s.weights()).to(dev)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        tl = P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid)
+        e1.record()
+        torch.cuda.synchronize()
+        tlq_ms += e0.elapsed_time(e1)
+        n_weights += s.N * s.K
+        R = None if s.rot != "dense" else bf16_dev(s.rotation_bf16()).to(dev)
+        kind = P.ROT_DENSE if s.rot == "dense" else P.ROT_HADAMARD
+        layers.append(P.QLayer(tl, s.N, s.K, kind, s.a_bits, s.had_block, R))
+        key = (s.K, s.n_salient) if args.config == 4 else (s.seed,)
+        if key not in x_cache:                       # the stack reuses one activation buffer per distinct K
+            xh = bf16_dev(s.activations()).pin_memory()
+            x_cache[key] = (xh, xh.to(dev))
+        Xs_host.append(x_cache[key][0])
+        Xs.append(x_cache[key][1])
+        del Wd
+    ydt = P.F32
+    y_cache = {}
+    for s in specs:                                   # outputs: one buffer per distinct N (reused across blocks)
+        key = s.N if args.config == 4 else s.seed
+        if key not in y_cache:
+            y_cache[key] = torch.empty((s.M, s.N), dtype=torch.float32, device=dev)
+        Ys.append(y_cache[key])
+    plan = P.StackPlan(layers, Xs, Ys, ydt)
+    ws = torch.empty(plan.need, dtype=torch.uint8, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        P.lrq_qlinear_stack(plan, ws, stream)
+
+    def timed(fn, n, flush_between=True):
+        evs = []
+        for _ in range(n):
+            if flush_between:
+                flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        flush.fill_(1); step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    ms = timed(step, args.steps)
+    barrier()
+    ms_step = float(np.mean(ms))
+
+    # ---- end to end: pinned host activations in, outputs back to pinned host memory, copies timed
+    uniq_x = {id(h): (h, d) for h, d in zip(Xs_host, Xs)}
+    uniq_y = {id(y): y for y in Ys}
+    y_host = {k: torch.empty(y.shape, dtype=y.dtype).pin_memory() for k, y in uniq_y.items()}
+    h2d = sum(h.numel() * 2 for h, _ in uniq_x.values())
+    d2h = sum(y.numel() * 4 for y in uniq_y.values())
+
+    def e2e_step():
+        for h, d in uniq_x.values():
+            d.copy_(h, non_blocking=True)
+        step()
+        for k, y in uniq_y.items():
+            y_host[k].copy_(y, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e2e_ms = float(np.mean(timed(e2e_step, max(2, min(args.steps, 10)))))
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+
+    if world > 1:
+        t = torch.tensor([ms_step, e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, e2e_ms = float(t[0]), float(t[1])
+
+    flops = layer_flops(specs)
+    tokens = sum(s.M for s in specs) / len(specs) if args.config != 4 else specs[0].M
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    e2e_val = world * flops / (e2e_ms * 1e-3) / 1e12
+
+    line = None
+    if rank == 0:
+        peaks = measured_peaks()
+        # ---- per-kernel roofline, measured live: the contraction (tensor bound) and rotate+quantize (HBM bound)
+        big = max(range(len(specs)), key=lambda i: specs[i].N * specs[i].K * specs[i].M)
+        s, L = specs[big], layers[big]
+        q, sc, zp = P.lrq_rotate_quantize_act(Xs[big], L.kind, s.a_bits, s.had_block, L.R)
+        gemm_ms = float(np.mean(timed(lambda: P.lrq_qgemm_codes(L, q, sc, zp, ydt, args.gemm_impl, Ys[big], stream), 20)))
+        gemm_tf = 2.0 * s.M * s.N * s.K / (gemm_ms * 1e-3) / 1e12
+        kbig = max(range(len(specs)), key=lambda i: specs[i].K * specs[i].M if specs[i].rot == "hadamard" else 0)
+        sr, Lr = specs[kbig], layers[kbig]
+        act_ws = torch.empty(256, dtype=torch.uint8, device=dev)
+        rot_ms = float(np.mean(timed(lambda: P.lrq_rotate_quantize_act(Xs[kbig], Lr.kind, sr.a_bits, sr.had_block,
+                                                                       Lr.R, workspace=act_ws, stream=stream), 20)))
+        rot_bytes = sr.M * (2.0 * sr.K + sr.K * sr.a_bits / 8.0 + 8.0)
+        rot_gbs = rot_bytes / (rot_ms * 1e-3) / 1e9
+        roofline = {"kernel": f"qgemm {s.name} {s.M}x{s.N}x{s.K} W{s.w_bits}A{s.a_bits}", "bound": "tensor",
+                    "achieved": gemm_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": gemm_tf / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"] + " burst bf16",
+                    "ms": gemm_ms}
+        roofline_rotq = {"kernel": f"rotq {sr.name} {sr.M}x{sr.K} B{sr.had_block} A{sr.a_bits}", "bound": "hbm",
+                         "achieved": rot_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rot_gbs / peaks["hbm_gbs"],
+                         "traffic": None, "peak_source": peaks["source"], "ms": rot_ms, "algorithmic_bytes": rot_bytes}
+        # ---- CPU baseline: the oracle, as it stands, on a bounded token sample
+        import oracle as orc
+        orc.build()
+        osp = specs[:4]
+        prepared = prepare_oracle(orc, osp, ORACLE_SAMPLE_TOKENS)
+        oracle_step(orc, prepared)
+        osec = float(np.mean([oracle_step(orc, prepared) for _ in range(3)]))
+        cpu_val = layer_flops(osp, ORACLE_SAMPLE_TOKENS) / osec / 1e12
+        n_rot_dense = sum(1 for s_ in specs if s_.rot == "dense")
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(args.config), "layers": len(specs), "out_dtype": "f32",
+                       "l2": "flushed between timed steps (512 MiB fill outside the timed events)",
+                       "parallelism": f"replicated batch x{world}, no collective"},
+            "tokens_per_s": world * tokens / (ms_step * 1e-3),
+            "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms},
+            "gpu_launches": args.steps * (2 * len(specs) + n_rot_dense),
+            "clocks": clocks, "roofline": roofline, "roofline_rotq": roofline_rotq,
+            "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+                             "sample": f"{ORACLE_SAMPLE_TOKENS} tokens of each of the first {len(osp)} linears (full K, N)",
+                             "tokens_per_s": ORACLE_SAMPLE_TOKENS / osec},
+            "tlq_weight_quantization": {"weights_per_s": n_weights / (tlq_ms * 1e-3), "ms": tlq_ms},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
+    ap.add_argument("--gemm-impl", type=int, default=0, choices=[0, 1],
+                    help="kernel timed alone for the roofline object: 0 tcgen05, 1 CUDA-core baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

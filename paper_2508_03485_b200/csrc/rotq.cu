@@ -155,7 +155,7 @@ static lrq_status launch_generic(bool f32, const void* X, int M, int K, long ldx
     const size_t smem = (size_t)K * sizeof(float);
     if (smem > 200 * 1024) return LRQ_ERR_UNSUPPORTED;
     auto kern = f32 ? rotq_generic_kernel<true> : rotq_generic_kernel<false>;
-    if (smem > 48 * 1024)
+    if (smem > 40 * 1024)
         LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int threads = (K >= 2048) ? 256 : (K >= 1024 ? 128 : 64);
     kern<<<M, threads, smem, st>>>(X, M, K, ldx, log2B, a_bits, mode, codes, scale, zp);

@@ -187,7 +187,7 @@ extern "C" lrq_status lrq_tlq_quantize_weights(const float* W_rot, int N, int K,
         grid.b[i] = i < grid.nb ? p->beta[i] : 0.0;
     }
     const size_t smem = (size_t)G * sizeof(double);
-    if (smem > 48 * 1024)
+    if (smem > 40 * 1024)
         LRQ_CUDA_TRY(cudaFuncSetAttribute(tlq_quantize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int threads = G >= 1024 ? 256 : 128;
     tlq_quantize_kernel<<<N, threads, smem, (cudaStream_t)cuda_stream>>>(W_rot, N, K, G, p->w_bits, p->integerize_I,

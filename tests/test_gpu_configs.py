@@ -39,11 +39,13 @@ def _run_layer(P, orc, spec, M=None):
     Rb = spec.rotation_bf16()
     Yo, oq, os_, oz = PU.oracle_layer_rows(orc, spec, xb[toks], T, Rb)
     Yg = Y[torch.from_numpy(toks).cuda()][:, torch.from_numpy(rows).cuda()].cpu().numpy()
-    fro, mabs = PU.check_out(Yg, Yo, spec.name)
-    # activation codes of the same call (from a separate lrq_rotate_quantize_act on the same input)
+    # activation codes of the same input through lrq_rotate_quantize_act (same kernels as inside lrq_qlinear)
     q, s, z = P.lrq_rotate_quantize_act(X, layer.kind, spec.a_bits, spec.had_block, layer.R)
     qn = PU.act_codes_to_numpy(q[torch.from_numpy(toks).cuda()], spec.a_bits)
-    frac, zf = PU.check_act(qn, s.cpu().numpy()[toks], z.cpu().numpy()[toks], oq, os_, oz, spec.name)
+    gz = z.cpu().numpy()[toks]
+    frac, zf = PU.check_act(qn, s.cpu().numpy()[toks], gz, oq, os_, oz, spec.name)
+    fro, mabs, nbound = PU.check_layer_out(orc, spec, T, Yg, qn, gz, Yo, oq, os_, oz, spec.name)
+    print(f"{spec.name}: rel_fro={fro:.2e} maxabs/rms={mabs:.2e} code_flips={frac:.2e} z_flips={zf} boundary_tokens={nbound}")
     layer.close()
     return fro, mabs, frac, zf
 
@@ -56,9 +58,10 @@ def test_config0_all_tokens(P, orc):
     Yo, oq, os_, oz = PU.oracle_layer_rows(orc, spec, xb, T)
     X = PU.bf16_to_device(xb)
     Y = P.lrq_qlinear(layer, X, P.F32)
-    PU.check_out(Y.cpu().numpy(), Yo, "cfg0")
     q, s, z = P.lrq_rotate_quantize_act(X, P.ROT_HADAMARD, 4, 1024)
-    PU.check_act(PU.act_codes_to_numpy(q, 4), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, "cfg0")
+    gq, gz = PU.act_codes_to_numpy(q, 4), z.cpu().numpy()
+    PU.check_act(gq, s.cpu().numpy(), gz, oq, os_, oz, "cfg0")
+    PU.check_layer_out(orc, spec, T, Y.cpu().numpy(), gq, gz, Yo, oq, os_, oz, "cfg0")
 
 
 @pytest.mark.parametrize("i", range(4))
