@@ -284,8 +284,9 @@ def run_cuda(args):
         kbig = max(range(len(specs)), key=lambda i: specs[i].K * specs[i].M if specs[i].rot == "hadamard" else 0)
         sr, Lr = specs[kbig], layers[kbig]
         act_ws = torch.empty(256, dtype=torch.uint8, device=dev)
+        rq = P.lrq_rotate_quantize_act(Xs[kbig], Lr.kind, sr.a_bits, sr.had_block, Lr.R)
         rot_ms = float(np.mean(timed(lambda: P.lrq_rotate_quantize_act(Xs[kbig], Lr.kind, sr.a_bits, sr.had_block,
-                                                                       Lr.R, workspace=act_ws, stream=stream), 20)))
+                                                                       Lr.R, workspace=act_ws, stream=stream, out=rq), 20)))
         rot_bytes = sr.M * (2.0 * sr.K + sr.K * sr.a_bits / 8.0 + 8.0)
         rot_gbs = rot_bytes / (rot_ms * 1e-3) / 1e9
         roofline = {"kernel": f"qgemm {s.name} {s.M}x{s.N}x{s.K} W{s.w_bits}A{s.a_bits}", "bound": "tensor",
@@ -328,6 +329,56 @@ def run_cuda(args):
     return line
 
 
+def run_kernel(args):
+    """Micro-benchmark of one kernel on one layer of the chosen workload (also the command the ncu captures
+    under profiles/ use): --kernel rotq | qgemm | tlq, --layer index, --tokens M override."""
+    import torch
+    import paper_2508_03485_b200 as P
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    s = config_layers(args.config)[args.layer]
+    M = args.tokens or s.M
+    grid = default_clip_grid()
+    stream = torch.cuda.current_stream()
+    Wd = torch.from_numpy(s.weights()).to(dev)
+    tl = P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid)
+    R = None if s.rot != "dense" else torch.from_numpy(s.rotation_bf16().view(np.int16)).view(torch.bfloat16).to(dev)
+    kind = P.ROT_DENSE if s.rot == "dense" else P.ROT_HADAMARD
+    L = P.QLayer(tl, s.N, s.K, kind, s.a_bits, s.had_block, R)
+    X = torch.from_numpy(s.activations(min(M, 4096)).view(np.int16)).view(torch.bfloat16).to(dev)
+    if M > X.shape[0]:
+        X = X.repeat((M + X.shape[0] - 1) // X.shape[0], 1)[:M].contiguous()
+    rq = P.lrq_rotate_quantize_act(X, kind, s.a_bits, s.had_block, R)
+    Y = torch.empty((M, s.N), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(256, L.workspace_bytes(M)), dtype=torch.uint8, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    if args.kernel == "rotq":
+        fn = lambda: P.lrq_rotate_quantize_act(X, kind, s.a_bits, s.had_block, R, workspace=ws, stream=stream, out=rq)
+        units, unit = M * (2.0 * s.K + s.K * s.a_bits / 8.0 + 8.0) / 1e9, "GB/s"
+    elif args.kernel == "qgemm":
+        fn = lambda: P.lrq_qgemm_codes(L, rq[0], rq[1], rq[2], P.F32, args.gemm_impl, Y, stream)
+        units, unit = 2.0 * M * s.N * s.K / 1e12, "TFLOP/s"
+    else:
+        fn = lambda: P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid)
+        units, unit = s.N * s.K / 1e9, "Gweights/s"
+    for _ in range(max(1, args.warmup)):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(args.steps):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); fn(); b.record(stream)
+        ts.append((a, b))
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in ts]
+    print(json.dumps({"kernel": args.kernel, "layer": s.name, "M": M, "K": s.K, "N": s.N, "rot": s.rot,
+                      "had_block": s.had_block, "w_bits": s.w_bits, "a_bits": s.a_bits,
+                      "ms_mean": float(np.mean(ms)), "ms_min": float(np.min(ms)),
+                      "rate_mean": units / (float(np.mean(ms)) * 1e-3), "rate_best": units / (float(np.min(ms)) * 1e-3),
+                      "unit": unit, "status": P.lrq_device_status()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -337,8 +388,13 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--gemm-impl", type=int, default=0, choices=[0, 1],
                     help="kernel timed alone for the roofline object: 0 tcgen05, 1 CUDA-core baseline")
+    ap.add_argument("--kernel", default=None, choices=["rotq", "qgemm", "tlq"], help="time one kernel only")
+    ap.add_argument("--layer", type=int, default=0, help="layer index of the workload for --kernel")
+    ap.add_argument("--tokens", type=int, default=0, help="override M for --kernel")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.kernel:
+        run_kernel(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)

@@ -147,7 +147,7 @@ def _act_params(kind: int, had_block: int, R: Optional[torch.Tensor], a_bits: in
 
 def lrq_rotate_quantize_act(X: torch.Tensor, kind: int, a_bits: int, had_block: int = 0,
                             R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM,
-                            workspace: Optional[torch.Tensor] = None, stream=None):
+                            workspace: Optional[torch.Tensor] = None, stream=None, out=None):
     """Rotation + per-token quantization (Eq. 12, Eq. 1) of device bf16 [M,K] activations.
     Returns (codes uint8, scale float32 [M], zero_point int32 [M])."""
     _need_cuda(X, R, workspace)
@@ -159,9 +159,13 @@ def lrq_rotate_quantize_act(X: torch.Tensor, kind: int, a_bits: int, had_block: 
     if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
         workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
     dev = X.device
-    codes = torch.empty((M, K * a_bits // 8), dtype=torch.uint8, device=dev)
-    scale = torch.empty((M,), dtype=torch.float32, device=dev)
-    zp = torch.empty((M,), dtype=torch.int32, device=dev)
+    if out is not None:
+        codes, scale, zp = out
+        assert codes.numel() == M * K * a_bits // 8 and scale.numel() == M and zp.numel() == M
+    else:
+        codes = torch.empty((M, K * a_bits // 8), dtype=torch.uint8, device=dev)
+        scale = torch.empty((M,), dtype=torch.float32, device=dev)
+        zp = torch.empty((M,), dtype=torch.int32, device=dev)
     wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
     rc = lib.lrq_rotate_quantize_act(_ptr(X), M, K, X.stride(0), C.byref(p), _ptr(codes), _ptr(scale), _ptr(zp),
                                      _ptr(workspace), wsb, _stream(stream))
