@@ -40,7 +40,7 @@ def check_act(gpu_q, gpu_s, gpu_z, orc_q, orc_s, orc_z, what="", flip_fraction=A
     gpu_q = np.asarray(gpu_q, dtype=np.int64)
     orc_q = np.asarray(orc_q, dtype=np.int64)
     gz, oz = np.asarray(gpu_z, dtype=np.int64), np.asarray(orc_z, dtype=np.int64)
-    assert np.allclose(np.asarray(gpu_s, dtype=np.float64), orc_s, rtol=2e-6, atol=0), f"{what}: scales differ"
+    assert np.allclose(np.asarray(gpu_s, dtype=np.float64), orc_s, rtol=2e-5, atol=0), f"{what}: scales differ"
     zflip = gz != oz
     assert np.abs(gz - oz).max() <= 1, f"{what}: zero-point off by more than one"
     assert zflip.sum() <= max(1, 0.01 * zflip.size), f"{what}: too many zero-point flips ({zflip.sum()})"
