@@ -115,6 +115,36 @@ lrq_status lrq_rotate_quantize_act(const void* X_bf16, int M, int K, long ldx, c
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * lrq_rotate_quantize_act for callers that cannot hand over device scratch.
+ *
+ * (The paper has no counterpart; this entry point exists for integration reasons only.)
+ *
+ * Some hosts of this library have no way to allocate device memory at the point where they call
+ * it: a plugin or a callback that runs inside someone else's pre-planned memory arena, a
+ * real-time or safety-reviewed inference loop in which cudaMalloc (which may synchronise the
+ * whole device and can fail) is forbidden after start-up, or a process whose allocator is owned
+ * by another runtime.  The dense rotation needs an fp32 scratch of M*K elements between the
+ * rotation GEMM and the quantizer; here that scratch is a fixed array inside the library image
+ * (LRQ_STATIC_SCRATCH_BYTES, held by every GPU that loads the library until the process exits).
+ *
+ *   - Arguments and results are those of lrq_rotate_quantize_act without the workspace pair.
+ *   - kind == LRQ_ROT_DENSE needs M*K*4 <= LRQ_STATIC_SCRATCH_BYTES, otherwise the call returns
+ *     LRQ_ERR_WORKSPACE and launches nothing (split the tokens into several calls).  The other
+ *     kinds use no scratch and have no size limit.
+ *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine).  The first
+ *     call on each device looks up the device address of the array (a host-side query, no launch);
+ *     make that first call before any stream capture.
+ *   - All calls on a device share the one array.  Its contents after a call are the last rotation's
+ *     output; nothing in it has to start at zero, because the rotation overwrites every element the
+ *     quantizer reads.  Two calls that may overlap on the GPU (different streams) race on it:
+ *     serialise them.
+ * ------------------------------------------------------------------------------------------- */
+#define LRQ_STATIC_SCRATCH_BYTES (8u << 20)
+
+lrq_status lrq_rotate_quantize_act_static(const void* X_bf16, int M, int K, long ldx, const lrq_act_params* p,
+                                          uint8_t* a_codes, float* a_scale, int32_t* a_zp, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * A quantized layer: TLQ codes, level tables and the activation recipe of one linear.
  * The handle is a small host object; it stores the device pointers it is given (it does not
  * copy or own them) and must be destroyed with lrq_layer_destroy.

@@ -20,8 +20,9 @@ _TORCH_DT = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16}
 EXPORTS = [
     "lrq_tlq_quantize_weights", "lrq_act_workspace_bytes", "lrq_rotate_quantize_act", "lrq_layer_create",
     "lrq_layer_destroy", "lrq_workspace_bytes", "lrq_qlinear", "lrq_qlinear_stack", "lrq_qgemm_codes",
-    "lrq_device_status", "lrq_status_string", "lrq_version",
+    "lrq_device_status", "lrq_status_string", "lrq_version", "lrq_rotate_quantize_act_static",
 ]
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class LrqError(RuntimeError):
@@ -60,6 +61,7 @@ def load_library() -> C.CDLL:
     lib.lrq_act_workspace_bytes.argtypes = [ci, ci, C.POINTER(_ActParams)]
     lib.lrq_act_workspace_bytes.restype = sz
     lib.lrq_rotate_quantize_act.argtypes = [vp, ci, ci, cl, C.POINTER(_ActParams), vp, vp, vp, vp, sz, vp]
+    lib.lrq_rotate_quantize_act_static.argtypes = [vp, ci, ci, cl, C.POINTER(_ActParams), vp, vp, vp, vp]
     lib.lrq_layer_create.argtypes = [C.POINTER(vp), ci, ci, ci, ci, vp, vp, vp, vp, vp, C.POINTER(_ActParams)]
     lib.lrq_layer_destroy.argtypes = [vp]
     lib.lrq_layer_destroy.restype = None
@@ -170,6 +172,29 @@ def lrq_rotate_quantize_act(X: torch.Tensor, kind: int, a_bits: int, had_block: 
     rc = lib.lrq_rotate_quantize_act(_ptr(X), M, K, X.stride(0), C.byref(p), _ptr(codes), _ptr(scale), _ptr(zp),
                                      _ptr(workspace), wsb, _stream(stream))
     _check(rc, "lrq_rotate_quantize_act")
+    return codes, scale, zp
+
+
+def lrq_rotate_quantize_act_static(X: torch.Tensor, kind: int, a_bits: int, had_block: int = 0,
+                                   R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM, stream=None, out=None):
+    """lrq_rotate_quantize_act for callers that cannot provide device scratch (a host that may not call
+    cudaMalloc once it is running, or whose memory is planned by another runtime): the dense rotation's
+    scratch is a fixed STATIC_SCRATCH_BYTES array inside the library.  ``out`` (codes, scale, zero_point)
+    lets such a caller pass its own pre-planned result buffers; without it this wrapper allocates them with
+    torch, the C entry point itself never allocates.  Raises LrqError (workspace) when M*K*4 exceeds the array."""
+    _need_cuda(X, R)
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    if out is not None:
+        codes, scale, zp = out
+    else:
+        codes = torch.empty((M, K * a_bits // 8), dtype=torch.uint8, device=X.device)
+        scale = torch.empty((M,), dtype=torch.float32, device=X.device)
+        zp = torch.empty((M,), dtype=torch.int32, device=X.device)
+    p = _act_params(kind, had_block, R, a_bits, mode)
+    rc = load_library().lrq_rotate_quantize_act_static(_ptr(X), M, K, X.stride(0), C.byref(p), _ptr(codes),
+                                                       _ptr(scale), _ptr(zp), _stream(stream))
+    _check(rc, "lrq_rotate_quantize_act_static")
     return codes, scale, zp
 
 

@@ -1,6 +1,7 @@
 // C-ABI entry points: argument checks, workspace carving, launches.  No entry point allocates
 // device memory or synchronises (lrq_device_status excepted, which reads one word back).
 #include "lrq_internal.cuh"
+#include <mutex>
 #include <new>
 
 // Status word written by a kernel whose bounded wait expired.  A file-scope device variable: in
@@ -60,6 +61,46 @@ extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long 
     }
     const int B = p->kind == LRQ_ROT_HADAMARD ? p->had_block : 1;
     return lrq_launch_rotq_hadamard(X, M, K, ldx, B, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Variant for callers that cannot allocate: the dense rotation's fp32 scratch is this fixed array.
+// In host code `g_static_scratch` is only a handle to the symbol; its address on the current device
+// comes from cudaGetSymbolAddress, queried once per device and cached.
+// ---------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[LRQ_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {};
+
+// Device address of the static scratch on the current device (nullptr on failure).
+void* static_scratch_address() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return nullptr; }
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+        g_scratch_addr[dev] = ptr;
+    }
+    return g_scratch_addr[dev];
+}
+}  // namespace
+
+extern "C" lrq_status lrq_rotate_quantize_act_static(const void* X, int M, int K, long ldx, const lrq_act_params* p,
+                                                     uint8_t* a_codes, float* a_scale, int32_t* a_zp,
+                                                     void* cuda_stream) {
+    if (!p) return LRQ_ERR_INVALID_ARG;
+    if (p->kind != LRQ_ROT_DENSE)                        // no scratch involved: the ordinary path, no workspace
+        return lrq_rotate_quantize_act(X, M, K, ldx, p, a_codes, a_scale, a_zp, nullptr, 0, cuda_stream);
+    if (M <= 0 || K <= 0) return LRQ_ERR_INVALID_ARG;
+    if ((size_t)M * (size_t)K * sizeof(float) > (size_t)LRQ_STATIC_SCRATCH_BYTES) return LRQ_ERR_WORKSPACE;
+    void* scratch = static_scratch_address();
+    if (!scratch) return LRQ_ERR_CUDA;
+    return lrq_rotate_quantize_act(X, M, K, ldx, p, a_codes, a_scale, a_zp, scratch, LRQ_STATIC_SCRATCH_BYTES,
+                                   cuda_stream);
 }
 
 extern "C" lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size,
