@@ -1,10 +1,175 @@
-// Outlier-aware rotation y = x . R (Sec. 4.2, Eq. 12, second case) as a dense contraction:
-// X bf16 [M,K] times R bf16 [K,K] into an fp32 scratch that the per-token quantizer then reads.
-// bf16 x bf16 products are exact in fp32; the sum is accumulated in fp32.
+// Outlier-aware rotation y = x . R (Sec. 4.2, Eq. 12, second case) as a dense contraction on the
+// 5th-generation tensor cores: X bf16 [M,K] times R bf16 [K,K] into an fp32 scratch that the
+// per-token quantizer then reads.  bf16 x bf16 products are exact in fp32; sums are accumulated in fp32.
+//
+// Persistent CTA per SM over 128 x 256 output tiles, 64-deep k-blocks, a 4-stage TMA pipeline:
+//   warp 0      one lane issues the TMA tile loads (X: K-major box 64 x 128; R: four 64 x 64 boxes, each
+//               64 output columns wide, one k-row per 128-byte line -> an MN-major UMMA operand)
+//   warp 1      allocates TMEM, one lane issues tcgen05.mma (M = 128, N = 256, K = 16) and commits
+//   warps 2-5   epilogue: tcgen05.ld of the finished accumulator, fp32 stores
+// The accumulator is double-buffered in TMEM (2 x 256 columns).  Every wait is bounded; on expiry the
+// CTA records a code in the status word, waits (bounded) for its TMA loads in flight and unwinds.
 #include "lrq_internal.cuh"
+#include "tc_ptx.cuh"
+#include <cuda.h>
 
 namespace {
+using namespace lrq_tc;
 
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;          // 16 KB
+constexpr int B_CHUNK_BYTES = BK * 128;             // 8 KB: 64 k-rows of 64 output columns
+constexpr int B_STAGE_BYTES = (BN / 64) * B_CHUNK_BYTES;   // 32 KB
+constexpr int STAGE_TX_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, EPI_WARP0 = 2, NUM_EPI_WARPS = 4;
+constexpr int NUM_THREADS = (EPI_WARP0 + NUM_EPI_WARPS) * 32;   // 192
+constexpr int TMEM_COLS = 512;
+
+struct __align__(8) Ctl {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + sizeof(Ctl);
+
+constexpr uint32_t IDESC = umma_idesc_bf16(BM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
+                  float* __restrict__ Y, int M, int K, int* status) {
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+    unsigned char* sA = base;
+    unsigned char* sB = base + STAGES * A_STAGE_BYTES;
+    Ctl* ctl = reinterpret_cast<Ctl*>(sB + STAGES * B_STAGE_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (M + BM - 1) / BM, tiles_n = (K + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int kblocks = (K + BK - 1) / BK;          // a ragged last k-block is zero-filled by TMA in both operands
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&ctl->tmem_full[b]), 1); mbar_init(smem_u32(&ctl->tmem_empty[b]), NUM_EPI_WARPS); }
+        ctl->abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tmX);
+        tma_prefetch_desc(&tmR);
+    }
+    if (warp == MMA_WARP) tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == PRODUCER_WARP) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, status, 11);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&ctl->full[s]);
+                    mbar_arrive_expect_tx(bar, STAGE_TX_BYTES);
+                    tma_load_2d(smem_u32(sA + s * A_STAGE_BYTES), &tmX, kb * BK, m0, bar);
+#pragma unroll
+                    for (int j = 0; j < BN / 64; ++j)
+                        tma_load_2d(smem_u32(sB + s * B_STAGE_BYTES + j * B_CHUNK_BYTES), &tmR, n0 + 64 * j, kb * BK, bar);
+                }
+            }
+            if (!ok) {
+                // loads already issued still write this CTA's shared memory: let each stage's last fill land
+                const uint32_t issued = it;
+                for (uint32_t back = 1; back <= (uint32_t)STAGES && back <= issued; ++back) {
+                    const uint32_t j = issued - back;
+                    const uint32_t bar = smem_u32(&ctl->full[j % STAGES]);
+                    for (uint32_t i = 0; i < kWaitLimit; ++i)
+                        if (mbar_try_wait(bar, (j / STAGES) & 1)) break;
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == MMA_WARP) {
+        if (lane == 0) {
+            uint32_t it = 0, t = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
+                const int buf = t & 1;
+                ok = mbar_wait(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, status, 12);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, status, 13);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(sA + s * A_STAGE_BYTES), b_addr = smem_u32(sB + s * B_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        tc_mma_f16(d_tmem,
+                                   umma_desc_sw128(a_addr + k * 32, 16, 1024),                    // 16 k = 32 bytes along the row
+                                   umma_desc_sw128(b_addr + k * 16 * 128, B_CHUNK_BYTES, 1024),   // 16 k = 16 rows of 128 bytes
+                                   IDESC, (kb | k) ? 1u : 0u);
+                    tc_commit(smem_u32(&ctl->empty[s]));
+                }
+                if (ok) tc_commit(smem_u32(&ctl->tmem_full[buf]));
+            }
+        }
+        __syncwarp();
+    } else {
+        const int ew = warp & 3;                         // TMEM lane quadrant this warp may read
+        const int row = ew * 32 + lane;
+        uint32_t t = 0;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
+            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+            const int buf = t & 1;
+            const int m = m0 + row;
+            const bool okw = mbar_wait(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, &ctl->abort_flag, status, 14);
+            tc_fence_after();
+            if (okw) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    if (n0 + c0 >= K) break;             // warp-uniform
+                    uint32_t acc[32];
+                    tc_ld32(tmem_base + ((uint32_t)(ew * 32) << 16) + (uint32_t)(buf * BN + c0), acc);
+                    tc_wait_ld();
+                    if (m < M) {
+                        float* dst = Y + (size_t)m * K + n0 + c0;
+                        if (n0 + c0 + 32 <= K) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                reinterpret_cast<uint4*>(dst)[j] = make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) if (n0 + c0 + j < K) dst[j] = __uint_as_float(acc[j]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[buf]));
+            if (ctl->abort_flag) break;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == MMA_WARP) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---- plain CUDA-core kernel for shapes the tensor-core kernel does not take ---------------------------
 constexpr int TM = 64, TN = 64, TK = 32;
 
 __global__ void __launch_bounds__(256)
@@ -49,9 +214,61 @@ rotgemm_simple_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ld
     }
 }
 
+// cuTensorMapEncodeTiled, fetched from the driver at first use (the library does not link libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            p = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// bf16 matrix [rows, cols] with `ld` elements between rows; box = box_cols x box_rows, 128-byte swizzle.
+bool make_map_bf16(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_cols,
+                   uint32_t box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y, cudaStream_t st) {
+    // TMA needs 16-byte aligned bases and row pitches; the fp32 rows are stored with 128-bit stores
+    const bool tc_ok = (K % 8) == 0 && (ldx % 8) == 0 && lrq_aligned(X, 16) && lrq_aligned(R, 16) && lrq_aligned(Y, 16);
+    if (tc_ok) {
+        CUtensorMap tmX, tmR;
+        if (!make_map_bf16(&tmX, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx, BK, BM)) return LRQ_ERR_CUDA;
+        if (!make_map_bf16(&tmR, R, (uint64_t)K, (uint64_t)K, (uint64_t)K, 64, BK)) return LRQ_ERR_CUDA;
+        static bool configured = false;
+        if (!configured) {
+            LRQ_CUDA_TRY(cudaFuncSetAttribute(rotgemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+            configured = true;
+        }
+        int dev = 0, sms = 0;
+        LRQ_CUDA_TRY(cudaGetDevice(&dev));
+        LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        const int tiles = ((M + BM - 1) / BM) * ((K + BN - 1) / BN);
+        rotgemm_tc_kernel<<<tiles < sms ? tiles : sms, NUM_THREADS, SMEM_BYTES, st>>>(tmX, tmR, Y, M, K, lrq_status_word());
+        LRQ_CUDA_TRY(cudaGetLastError());
+        return LRQ_OK;
+    }
     dim3 grid((K + TN - 1) / TN, (M + TM - 1) / TM), block(256);
     rotgemm_simple_kernel<<<grid, block, 0, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx,
                                                   static_cast<const __nv_bfloat16*>(R), Y);
