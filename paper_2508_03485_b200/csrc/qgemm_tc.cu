@@ -7,113 +7,70 @@
 // integer below 256, so both operands are exactly bf16 numbers; products are exact and only the
 // fp32 accumulation order differs from the fp64 definition.
 //
-// One persistent CTA per SM walks over 128 x 256 output tiles.  Warp roles:
-//   warps 0-3   expand activation codes of the tile's 128 tokens into the bf16 A stage
-//   warps 4-11  decode TLQ codes of the tile's 256 output channels through the row's level table
-//               (held in registers as two byte planes, looked up with byte permutes) into the B stage
-//   warps 12-15 epilogue: tcgen05.ld the finished accumulator, scale, store
-//   warp  16    allocates TMEM and issues tcgen05.mma (one elected lane)
-// The A/B stages use the canonical K-major 128-byte-swizzled layout that the UMMA shared-memory
-// descriptor expects; they are written with ordinary shared stores, published to the async proxy
-// with fence.proxy.async and handed over through mbarriers.  The accumulator is double-buffered in
-// TMEM (2 x 256 columns) so that the epilogue of one tile overlaps the main loop of the next.
-// Every wait is bounded: when one expires the CTA records a code in the status word, stops waiting
-// and runs to its end (TMEM is always freed).
+// The decode of both operands runs on the integer ALUs and is what bounds the kernel, so the tile is
+// shaped to decode each element as rarely as possible: a pair of CTAs (a cluster of two, cta_group::2)
+// owns a 256 x 256 output tile.  Each CTA decodes its own 128 token rows of A and only its own 128 of
+// the 256 weight rows of B; the tensor core reads the other half from the peer's shared memory.
+// Per CTA (18 warps):
+//   warp 0       one lane streams the packed code tiles (128 rows x 64 codes of each operand per k-block)
+//                into shared memory with TMA, CSTAGES deep
+//   warp 1       allocates TMEM; in the even CTA one lane issues tcgen05.mma (M = 256, N = 256, K = 16)
+//   warps 2-9    decode TLQ weight codes through the row's level table (held in registers as two byte
+//                planes, looked up with byte permutes) into the bf16 B stage
+//   warps 10-13  expand activation codes into the bf16 A stage
+//   warps 14-17  epilogue: tcgen05.ld the finished accumulator, scale, store
+// The bf16 stages use the canonical K-major 128-byte-swizzled UMMA layout; they are written with
+// ordinary shared stores, published to the async proxy with fence.proxy.async and handed to the MMA
+// thread of the even CTA through an mbarrier there (in the odd CTA the decode warps arrive on a local
+// barrier and one relay thread forwards each completed stage with a single cluster-scope arrival).  Stage release and
+// accumulator completion come back to both CTAs through multicast tcgen05.commit.  The accumulator is
+// double-buffered in TMEM (2 x 256 columns) so that the epilogue of one tile overlaps the main loop of
+// the next.  Every wait is bounded: when one expires the CTA records a code in the status word, stops
+// waiting, lets its TMA loads land, and both CTAs meet at the final cluster barrier (TMEM is always freed).
 //
-// To keep the expansion cheap the A operand carries a constant offset that the epilogue removes:
-// 8-bit codes are fed as q - 128, 4-bit codes as q - 8 (the zero-point term absorbs it); centring
-// also keeps the accumulator free of a large common-mode term.
+// The A operand carries a constant offset that the epilogue removes: 8-bit codes are fed as q - 128,
+// 4-bit codes as q - 8 (the zero-point term absorbs it); centring keeps the expansion cheap and the
+// accumulator free of a large common-mode term.
 #include "lrq_internal.cuh"
+#include "tc_ptx.cuh"
+#include "tma_host.cuh"
 
 namespace {
+using namespace lrq_tc;
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int STAGES = 4;
-constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
-constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KB
-constexpr int NUM_A_WARPS = 4, NUM_B_WARPS = 8, NUM_EPI_WARPS = 4;
-constexpr int EPI_WARP0 = NUM_A_WARPS + NUM_B_WARPS;          // 12 (a multiple of 4: TMEM lane quadrants line up)
-constexpr int MMA_WARP = EPI_WARP0 + NUM_EPI_WARPS;           // 16
-constexpr int NUM_THREADS = (MMA_WARP + 1) * 32;              // 544
+constexpr int BM_CTA = 128;                  // token rows per CTA; the pair's tile has 256
+constexpr int BN = 256;                      // output channels per tile
+constexpr int BN_CTA = 128;                  // weight rows decoded per CTA
+constexpr int BK = 64;
+constexpr int STAGES = 4;                    // bf16 operand stages
+constexpr int CSTAGES = 4;                   // packed-code stages
+constexpr int A_STAGE_BYTES = BM_CTA * BK * 2;      // 16 KB
+constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;      // 16 KB
+constexpr int AC_STAGE_BYTES = BM_CTA * BK;         // room for 8-bit codes (4-bit codes use half)
+constexpr int WC_STAGE_BYTES = BN_CTA * BK / 2;     // 4 KB
+constexpr int TMA_WARP = 0, MMA_WARP = 1, B_WARP0 = 2, NUM_B_WARPS = 8, A_WARP0 = 10, NUM_A_WARPS = 4;
+constexpr int EPI_WARP0 = 14, NUM_EPI_WARPS = 4;
+constexpr int NUM_DEC_WARPS = NUM_A_WARPS + NUM_B_WARPS;
+constexpr int NUM_THREADS = (EPI_WARP0 + NUM_EPI_WARPS) * 32;      // 576
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct __align__(8) SharedCtl {
-    uint64_t full[STAGES];
-    uint64_t empty[STAGES];
-    uint64_t tmem_full[2];
-    uint64_t tmem_empty[2];
+    uint64_t cfull[CSTAGES];      // code stage filled by TMA                       (local)
+    uint64_t cempty[CSTAGES];     // code stage read by every decode warp           (local)
+    uint64_t full[STAGES];        // bf16 stage written: own decode warps (+ the peer's relay, even CTA)
+    uint64_t empty[STAGES];       // bf16 stage consumed by the MMAs                (each CTA, multicast commit)
+    uint64_t tmem_full[2];        // accumulator complete                           (each CTA, multicast commit)
+    uint64_t tmem_empty[2];       // accumulator drained by both CTAs' epilogues    (used in the even CTA)
     uint32_t tmem_base;
     volatile int abort_flag;
     float col[2][3][BN];          // per TMEM buffer: wsum, wscale, bias of the tile's columns
 };
 
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + sizeof(SharedCtl);
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
+                              (size_t)CSTAGES * (AC_STAGE_BYTES + WC_STAGE_BYTES) + sizeof(SharedCtl);
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false (and raises the CTA's abort flag) if the phase never completed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, SharedCtl* ctl, int* status, int code) {
-    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (ctl->abort_flag) return false;
-    }
-    ctl->abort_flag = 1;
-    if (status) atomicCAS(status, 0, code);
-    return false;
-}
-
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// UMMA shared-memory descriptor: K-major operand, 128-byte swizzle, rows of 64 bf16 (128 B), groups of
-// 8 rows 1024 B apart.  Bits: [0,14) address>>4, [16,30) leading offset>>4 (unused for this layout),
-// [32,46) stride offset>>4, [46,48) descriptor version 1, [61,64) layout type 2 (128B swizzle).
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-// Instruction descriptor, kind::f16: fp32 accumulator (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
-// both K-major (bits 15, 16 = 0), N>>3 at bits 17-22, M>>4 at bits 24-28.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t IDESC = umma_idesc_bf16(2 * BM_CTA, BN, false, false);
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     uint32_t d;
@@ -151,22 +108,19 @@ __device__ __forceinline__ void expand_a4(uint32_t w, uint32_t* o) {
 // The table is kept as two byte planes (low and high byte of each bf16 entry), 16 entries = 4 + 4 registers.
 struct Lut { uint32_t lo[4], hi[4]; };
 
+// Levels are exact bf16 numbers stored as fp32: the upper two bytes of each word are the entry.
 template <int W_BITS>
-__device__ __forceinline__ void load_lut(Lut& L, const float* __restrict__ tab) {
-    constexpr int NL = 1 << W_BITS;
-    uint32_t e[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) e[i] = 0;
-#pragma unroll
-    for (int i = 0; i < NL / 4; ++i) {
-        const float4 v = *reinterpret_cast<const float4*>(tab + 4 * i);
-        e[4 * i] = __float_as_uint(v.x) >> 16; e[4 * i + 1] = __float_as_uint(v.y) >> 16;   // levels are exact bf16 numbers
-        e[4 * i + 2] = __float_as_uint(v.z) >> 16; e[4 * i + 3] = __float_as_uint(v.w) >> 16;
-    }
+__device__ __forceinline__ void build_lut(Lut& L, const float4* raw) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        L.lo[j] = (e[4 * j] & 0xFF) | ((e[4 * j + 1] & 0xFF) << 8) | ((e[4 * j + 2] & 0xFF) << 16) | ((e[4 * j + 3] & 0xFF) << 24);
-        L.hi[j] = (e[4 * j] >> 8) | ((e[4 * j + 1] >> 8) << 8) | ((e[4 * j + 2] >> 8) << 16) | ((e[4 * j + 3] >> 8) << 24);
+        if (j < (1 << W_BITS) / 4) {
+            const uint32_t t01 = prmt(__float_as_uint(raw[j].x), __float_as_uint(raw[j].y), 0x7632u);
+            const uint32_t t23 = prmt(__float_as_uint(raw[j].z), __float_as_uint(raw[j].w), 0x7632u);
+            L.lo[j] = prmt(t01, t23, 0x6420u);
+            L.hi[j] = prmt(t01, t23, 0x7531u);
+        } else {
+            L.lo[j] = 0; L.hi[j] = 0;
+        }
     }
 }
 
@@ -192,144 +146,243 @@ __device__ __forceinline__ void decode_w(uint32_t w, const Lut& L, uint32_t* o) 
     }
 }
 
+// Named barrier 1 over the epilogue warps, returning the OR of `pred` over all of them.
+__device__ __forceinline__ bool bar_or_epilogue(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\n"
+        "bar.red.or.pred p, 1, %2, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(r) : "r"((uint32_t)pred), "n"(NUM_EPI_WARPS * 32) : "memory");
+    return r != 0;
+}
+
 __device__ __forceinline__ void sts128(unsigned char* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
 }
 
 struct Params {
-    const uint8_t* a_codes; const float* a_scale; const int32_t* a_zp;
-    const uint8_t* w_codes; const float* levels; const float* wsum; const float* wscale; const float* bias;
+    const float* a_scale; const int32_t* a_zp;
+    const float* levels; const float* wsum; const float* wscale; const float* bias;
     void* Y; long ldy; int M, N, K, G, y_dtype; int* status;
 };
 
 template <int A_BITS, int W_BITS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-qgemm_tc_kernel(const Params p) {
+qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-    unsigned char* sA = base;                                   // STAGES x 16 KB
-    unsigned char* sB = base + STAGES * A_STAGE_BYTES;          // STAGES x 32 KB
-    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(sB + STAGES * B_STAGE_BYTES);
+    unsigned char* sA = base;                                       // STAGES x 16 KB
+    unsigned char* sB = sA + STAGES * A_STAGE_BYTES;                // STAGES x 16 KB
+    unsigned char* sAc = sB + STAGES * B_STAGE_BYTES;               // CSTAGES x 8 KB
+    unsigned char* sWc = sAc + CSTAGES * AC_STAGE_BYTES;            // CSTAGES x 4 KB
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(sWc + CSTAGES * WC_STAGE_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const uint32_t rank = cluster_ctarank();                       // 0: issues the MMAs, 1: its peer
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int tiles_m = (p.M + 2 * BM_CTA - 1) / (2 * BM_CTA), tiles_n = (p.N + BN - 1) / BN;
     const int num_tiles = tiles_m * tiles_n;
     const int kblocks = p.K / BK;
     constexpr int NLEV = 1 << W_BITS;
+    constexpr int AC_ROW_BYTES = BK * A_BITS / 8;                   // 64 or 32 code bytes per token and k-block
+    constexpr uint32_t CODE_TX_BYTES = BM_CTA * AC_ROW_BYTES + WC_STAGE_BYTES;
 
     if (threadIdx.x == 0) {
+        for (int s = 0; s < CSTAGES; ++s) {
+            mbar_init(smem_u32(&ctl->cfull[s]), 1);
+            mbar_init(smem_u32(&ctl->cempty[s]), NUM_DEC_WARPS);
+        }
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), NUM_A_WARPS + NUM_B_WARPS);
+            mbar_init(smem_u32(&ctl->full[s]), rank == 0 ? NUM_DEC_WARPS + 1 : NUM_DEC_WARPS);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[b]), NUM_EPI_WARPS);
+            mbar_init(smem_u32(&ctl->tmem_empty[b]), 2 * NUM_EPI_WARPS);
         }
         ctl->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_init_fence();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmW);
     }
-    if (warp == MMA_WARP) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == MMA_WARP) tmem_alloc_pair(smem_u32(&ctl->tmem_base), TMEM_COLS);
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                       // the peer's barriers exist before anyone arrives on them
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (warp < NUM_A_WARPS) {
-        // =============================== A producers: one token row per thread ===============================
-        const int r = threadIdx.x;                                // 0..127
-        constexpr int ROW_BYTES = BK * A_BITS / 8;                // 64 (8-bit) or 32 (4-bit) code bytes per k-block
-        constexpr int NV = ROW_BYTES / 16;
-        uint32_t it = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-            const int m0 = (tile % tiles_m) * BM;
-            const int m = min(m0 + r, p.M - 1);                   // rows past M read a valid row; never stored
-            const uint4* src = reinterpret_cast<const uint4*>(p.a_codes + (size_t)m * ((size_t)p.K * A_BITS / 8));
-            uint4 cur[NV];
-#pragma unroll
-            for (int i = 0; i < NV; ++i) cur[i] = __ldg(src + i);
-            for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                uint4 nxt[NV];
-                if (kb + 1 < kblocks) {
-#pragma unroll
-                    for (int i = 0; i < NV; ++i) nxt[i] = __ldg(src + (size_t)(kb + 1) * NV + i);
+    if (warp == TMA_WARP) {
+        // =============================== packed codes: global -> shared (TMA) ===============================
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                const int m_base = (tile % tiles_m) * 2 * BM_CTA + (int)rank * BM_CTA;
+                const int n_base = (tile / tiles_m) * BN + (int)rank * BN_CTA;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int cs = it % CSTAGES;
+                    ok = mbar_wait(smem_u32(&ctl->cempty[cs]), ((it / CSTAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 1);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&ctl->cfull[cs]);
+                    mbar_arrive_expect_tx(bar, CODE_TX_BYTES);
+                    tma_load_2d(smem_u32(sAc + cs * AC_STAGE_BYTES), &tmA, kb * AC_ROW_BYTES, m_base, bar);
+                    tma_load_2d(smem_u32(sWc + cs * WC_STAGE_BYTES), &tmW, kb * (BK / 2), n_base, bar);
                 }
-                const int s = it % STAGES;
-                if (!mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, ctl, p.status, 1)) break;
-                unsigned char* dst = sA + s * A_STAGE_BYTES;
-                if (A_BITS == 8) {
-#pragma unroll
-                    for (int i = 0; i < NV; ++i) {                // 16 codes -> two 16-byte chunks
-                        uint32_t o[8];
-                        expand_a8(cur[i].x, o[0], o[1]); expand_a8(cur[i].y, o[2], o[3]);
-                        expand_a8(cur[i].z, o[4], o[5]); expand_a8(cur[i].w, o[6], o[7]);
-                        sts128(dst + swz(r, 2 * i), o[0], o[1], o[2], o[3]);
-                        sts128(dst + swz(r, 2 * i + 1), o[4], o[5], o[6], o[7]);
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < NV; ++i) {                // 32 codes -> four chunks
-                        uint32_t o[4];
-                        expand_a4(cur[i].x, o); sts128(dst + swz(r, 4 * i), o[0], o[1], o[2], o[3]);
-                        expand_a4(cur[i].y, o); sts128(dst + swz(r, 4 * i + 1), o[0], o[1], o[2], o[3]);
-                        expand_a4(cur[i].z, o); sts128(dst + swz(r, 4 * i + 2), o[0], o[1], o[2], o[3]);
-                        expand_a4(cur[i].w, o); sts128(dst + swz(r, 4 * i + 3), o[0], o[1], o[2], o[3]);
-                    }
-                }
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
-#pragma unroll
-                for (int i = 0; i < NV; ++i) cur[i] = nxt[i];
             }
-            if (ctl->abort_flag) break;
+            if (!ok) {     // loads already issued still write this CTA's shared memory: let them land
+                for (uint32_t back = 1; back <= (uint32_t)CSTAGES && back <= it; ++back) {
+                    const uint32_t j = it - back;
+                    const uint32_t bar = smem_u32(&ctl->cfull[j % CSTAGES]);
+                    for (uint32_t i = 0; i < kWaitLimit; ++i)
+                        if (mbar_try_wait(bar, (j / CSTAGES) & 1)) break;
+                }
+            }
         }
-    } else if (warp < EPI_WARP0) {
-        // =============================== B producers: one output channel per thread ==========================
-        const int r = threadIdx.x - NUM_A_WARPS * 32;             // 0..255
+        __syncwarp();
+    } else if (warp == MMA_WARP) {
+        // =============================== MMA issuer (even CTA only) ========================================
+        if (rank == 0 && lane == 0) {
+            uint32_t it = 0, t = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++t) {
+                const int buf = t & 1;
+                ok = mbar_wait_cluster(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, p.status, 4);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    ok = mbar_wait_cluster(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, p.status, 5);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(sA + s * A_STAGE_BYTES), b_addr = smem_u32(sB + s * B_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        tc_mma_f16_pair(d_tmem, umma_desc_sw128(a_addr + k * 32, 16, 1024),
+                                        umma_desc_sw128(b_addr + k * 32, 16, 1024), IDESC, (kb | k) ? 1u : 0u);
+                    tc_commit_pair(smem_u32(&ctl->empty[s]), 3);        // both CTAs may refill the stage
+                }
+                if (ok) tc_commit_pair(smem_u32(&ctl->tmem_full[buf]), 3);   // accumulator complete, both halves
+            }
+        } else if (rank == 1 && lane == 0) {
+            // relay: once this CTA's decode warps have all published a stage, tell the even CTA with one
+            // cluster-scope release (the decode warps themselves only pay for CTA-scope arrivals)
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, p.status, 9);
+                    if (!ok) break;
+                    mbar_arrive_cluster(smem_u32(&ctl->full[s]), 0);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp < A_WARP0) {
+        // =============================== B decode: 32 codes of one weight row per thread ====================
+        const int t = threadIdx.x - B_WARP0 * 32;                  // 0..255
+        const int row = t >> 1, c = t & 1;                         // row of the CTA's 128, half of the k-block
         const int ngrp = p.K / p.G, kb_per_grp = p.G / BK;
         uint32_t it = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-            const int n0 = (tile / tiles_m) * BN;
-            const int n = min(n0 + r, p.N - 1);
-            const uint4* src = reinterpret_cast<const uint4*>(p.w_codes + (size_t)n * (p.K / 2));
-            const float* tab = p.levels + (size_t)n * ngrp * NLEV;
+        for (int tile = pair; tile < num_tiles; tile += num_pairs) {
+            const int n_base = (tile / tiles_m) * BN + (int)rank * BN_CTA;
+            const int n = min(n_base + row, p.N - 1);               // rows past N decode a valid table; never stored
+            const float4* tab = reinterpret_cast<const float4*>(p.levels + (size_t)n * ngrp * NLEV);
             Lut L;
-            uint4 cur[2];
-            cur[0] = __ldg(src); cur[1] = __ldg(src + 1);
+            float4 raw[NLEV / 4];
+#pragma unroll
+            for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + j);
+            bool ok = true;
             for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                uint4 nxt[2];
-                if (kb + 1 < kblocks) { nxt[0] = __ldg(src + 2 * (kb + 1)); nxt[1] = __ldg(src + 2 * (kb + 1) + 1); }
-                if (kb % kb_per_grp == 0) load_lut<W_BITS>(L, tab + (size_t)(kb / kb_per_grp) * NLEV);
+                if (kb % kb_per_grp == 0) {
+                    build_lut<W_BITS>(L, raw);
+                    const int g1 = kb / kb_per_grp + 1;            // fetch the next group's table a group ahead
+                    if (g1 < ngrp) {
+#pragma unroll
+                        for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)g1 * (NLEV / 4) + j);
+                    }
+                }
+                const int cs = it % CSTAGES;
+                ok = mbar_wait_warp(smem_u32(&ctl->cfull[cs]), (it / CSTAGES) & 1, &ctl->abort_flag, p.status, 2);
+                if (!ok) break;
+                const uint4 cw = *reinterpret_cast<const uint4*>(sWc + cs * WC_STAGE_BYTES + t * 16);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->cempty[cs]));
+                uint32_t o[16];
+                decode_w<W_BITS>(cw.x, L, o); decode_w<W_BITS>(cw.y, L, o + 4);
+                decode_w<W_BITS>(cw.z, L, o + 8); decode_w<W_BITS>(cw.w, L, o + 12);
                 const int s = it % STAGES;
-                if (!mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, ctl, p.status, 2)) break;
+                ok = mbar_wait_warp(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 3);
+                if (!ok) break;
                 unsigned char* dst = sB + s * B_STAGE_BYTES;
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    uint32_t o[4];
-                    decode_w<W_BITS>(cur[i].x, L, o); sts128(dst + swz(r, 4 * i), o[0], o[1], o[2], o[3]);
-                    decode_w<W_BITS>(cur[i].y, L, o); sts128(dst + swz(r, 4 * i + 1), o[0], o[1], o[2], o[3]);
-                    decode_w<W_BITS>(cur[i].z, L, o); sts128(dst + swz(r, 4 * i + 2), o[0], o[1], o[2], o[3]);
-                    decode_w<W_BITS>(cur[i].w, L, o); sts128(dst + swz(r, 4 * i + 3), o[0], o[1], o[2], o[3]);
+                for (int j = 0; j < 4; ++j) sts128(dst + swz(row, 4 * c + j), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
+            }
+            if (!ok || __any_sync(0xffffffffu, ctl->abort_flag != 0)) break;
+        }
+    } else if (warp < EPI_WARP0) {
+        // =============================== A expansion: 16-byte chunks of the code stage ======================
+        const int t = threadIdx.x - A_WARP0 * 32;                  // 0..127
+        constexpr int TASKS = BM_CTA * AC_ROW_BYTES / 16 / (NUM_A_WARPS * 32);   // 4 (8-bit) or 2 (4-bit)
+        constexpr int CH_PER_ROW = AC_ROW_BYTES / 16;              // 4 or 2 code chunks per token row
+        uint32_t it = 0;
+        for (int tile = pair; tile < num_tiles; tile += num_pairs) {
+            bool ok = true;
+            for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                const int cs = it % CSTAGES;
+                ok = mbar_wait_warp(smem_u32(&ctl->cfull[cs]), (it / CSTAGES) & 1, &ctl->abort_flag, p.status, 6);
+                if (!ok) break;
+                uint4 cw[TASKS];
+#pragma unroll
+                for (int i = 0; i < TASKS; ++i)
+                    cw[i] = *reinterpret_cast<const uint4*>(sAc + cs * AC_STAGE_BYTES + (i * NUM_A_WARPS * 32 + t) * 16);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->cempty[cs]));
+                uint32_t o[TASKS][A_BITS == 8 ? 8 : 16];
+#pragma unroll
+                for (int i = 0; i < TASKS; ++i) {
+                    if constexpr (A_BITS == 8) {
+                        expand_a8(cw[i].x, o[i][0], o[i][1]); expand_a8(cw[i].y, o[i][2], o[i][3]);
+                        expand_a8(cw[i].z, o[i][4], o[i][5]); expand_a8(cw[i].w, o[i][6], o[i][7]);
+                    } else {
+                        expand_a4(cw[i].x, o[i]); expand_a4(cw[i].y, o[i] + 4);
+                        expand_a4(cw[i].z, o[i] + 8); expand_a4(cw[i].w, o[i] + 12);
+                    }
+                }
+                const int s = it % STAGES;
+                ok = mbar_wait_warp(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 7);
+                if (!ok) break;
+                unsigned char* dst = sA + s * A_STAGE_BYTES;
+#pragma unroll
+                for (int i = 0; i < TASKS; ++i) {
+                    const int id = i * NUM_A_WARPS * 32 + t;
+                    const int row = id / CH_PER_ROW, cc = id % CH_PER_ROW;
+                    constexpr int OUT_CH = 8 / CH_PER_ROW;         // bf16 chunks per code chunk: 2 or 4
+#pragma unroll
+                    for (int j = 0; j < OUT_CH; ++j)
+                        sts128(dst + swz(row, OUT_CH * cc + j), o[i][4 * j], o[i][4 * j + 1], o[i][4 * j + 2], o[i][4 * j + 3]);
                 }
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
-                cur[0] = nxt[0]; cur[1] = nxt[1];
             }
-            if (ctl->abort_flag) break;
+            if (!ok || __any_sync(0xffffffffu, ctl->abort_flag != 0)) break;
         }
-    } else if (warp < MMA_WARP) {
+    } else {
         // =============================== epilogue: TMEM -> registers -> global ===============================
-        const int ew = warp - EPI_WARP0;                           // TMEM lane quadrant
-        const int et = threadIdx.x - EPI_WARP0 * 32;               // 0..127 = accumulator row
-        const float zoff = (A_BITS == 8) ? 128.f : 8.f;      // the A operand is fed as q - 128 / q - 8
+        const int ew = warp & 3;                                   // TMEM lane quadrant this warp may read
+        const int et = threadIdx.x - EPI_WARP0 * 32;               // 0..127, for the cooperative column staging
+        const int row = ew * 32 + lane;                            // accumulator row within the CTA
+        const float zoff = (A_BITS == 8) ? 128.f : 8.f;            // the A operand is fed as q - 128 / q - 8
         uint32_t t = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++t) {
-            const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
+            const int m0 = (tile % tiles_m) * 2 * BM_CTA + (int)rank * BM_CTA, n0 = (tile / tiles_m) * BN;
             const int buf = t & 1;
             // stage the tile's per-column terms (wsum, wscale, bias) in shared memory
             float (*col)[BN] = ctl->col[buf];
@@ -340,12 +393,13 @@ qgemm_tc_kernel(const Params p) {
                 col[1][c] = (ok && p.wscale) ? __ldg(p.wscale + n) : 1.f;
                 col[2][c] = (ok && p.bias) ? __ldg(p.bias + n) : 0.f;
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
-            const int m = m0 + et;
+            // barrier over the four epilogue warps; they leave together once any of them has seen the abort flag
+            if (bar_or_epilogue(ctl->abort_flag != 0)) break;
+            const int m = m0 + row;
             const bool row_ok = m < p.M;
             const float sm = row_ok ? __ldg(p.a_scale + m) : 0.f;
             const float zm = row_ok ? (float)__ldg(p.a_zp + m) + zoff : 0.f;
-            const bool okw = mbar_wait(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, ctl, p.status, 3);
+            const bool okw = mbar_wait_warp(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, &ctl->abort_flag, p.status, 8);
             tc_fence_after();
             if (okw) {
 #pragma unroll 1
@@ -397,56 +451,44 @@ qgemm_tc_kernel(const Params p) {
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[buf]));
-            if (ctl->abort_flag) break;
+            if (lane == 0) mbar_arrive_cluster(smem_u32(&ctl->tmem_empty[buf]), 0);
         }
-    } else {
-        // =============================== MMA issuer ==========================================================
-        if (lane == 0) {
-            uint32_t it = 0, t = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
-                const int buf = t & 1;
-                ok = mbar_wait(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, ctl, p.status, 4);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    ok = mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1, ctl, p.status, 5);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t a_addr = smem_u32(sA + s * A_STAGE_BYTES), b_addr = smem_u32(sB + s * B_STAGE_BYTES);
-#pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        tc_mma_bf16(d_tmem, make_desc(a_addr + k * 32), make_desc(b_addr + k * 32), IDESC, (kb | k) ? 1u : 0u);
-                    tc_commit(smem_u32(&ctl->empty[s]));            // stage reusable once these MMAs have read it
-                }
-                if (ok) tc_commit(smem_u32(&ctl->tmem_full[buf]));  // accumulator complete
-            }
-        }
-        __syncwarp();
     }
 
-    // teardown: every role has left its loop; nothing is waiting any more
+    // teardown: every role has left its loop.  Neither CTA may exit (or release TMEM) while its peer can
+    // still arrive on its barriers or have MMAs reading its shared memory.
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();
     if (warp == MMA_WARP) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 
 template <int A_BITS, int W_BITS>
-lrq_status launch(const Params& p, int grid, cudaStream_t st) {
+lrq_status launch(const Params& p, const CUtensorMap& tmA, const CUtensorMap& tmW, int num_tiles, cudaStream_t st) {
     auto kern = qgemm_tc_kernel<A_BITS, W_BITS>;
-    static bool configured = false;
-    if (!configured) {
+    static int max_pairs = 0;                 // per process; the library targets identical GPUs
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (!max_pairs) {
         LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-        configured = true;
+        int dev = 0, sms = 0, clusters = 0;
+        LRQ_CUDA_TRY(cudaGetDevice(&dev));
+        LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        cfg.gridDim = dim3(sms & ~1);
+        LRQ_CUDA_TRY(cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg));
+        if (clusters < 1) return LRQ_ERR_CUDA;
+        max_pairs = clusters < sms / 2 ? clusters : sms / 2;
     }
-    kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(p);
-    LRQ_CUDA_TRY(cudaGetLastError());
+    const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
+    cfg.gridDim = dim3(2 * pairs);
+    LRQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p, tmA, tmW));
     return LRQ_OK;
 }
 
@@ -454,25 +496,26 @@ lrq_status launch(const Params& p, int grid, cudaStream_t st) {
 
 lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                                const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st) {
-    // shapes this kernel takes: whole 64-wide k-blocks that never straddle a TLQ group; 16-byte code rows
+    // shapes this kernel takes: whole 64-wide k-blocks that never straddle a TLQ group; 16-byte aligned code rows
     if (L->K % BK || L->group % BK) return LRQ_ERR_UNSUPPORTED;
     if (L->w_bits < 3 || L->w_bits > 4) return LRQ_ERR_UNSUPPORTED;   // 2-bit tables take the CUDA-core kernel
-    if (!lrq_aligned(L->levels, 16) || !lrq_aligned(L->codes, 16)) return LRQ_ERR_UNSUPPORTED;
+    if (!lrq_aligned(L->levels, 16) || !lrq_aligned(L->codes, 16) || !lrq_aligned(a_codes, 16)) return LRQ_ERR_UNSUPPORTED;
     const size_t es = dt == LRQ_F32 ? 4 : 2;
     if (!lrq_aligned(Y, 16) || ((size_t)ldy * es) % 16) return LRQ_ERR_UNSUPPORTED;
-    int dev = 0, sms = 0;
-    LRQ_CUDA_TRY(cudaGetDevice(&dev));
-    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int ab = L->act.a_bits;
     Params p;
-    p.a_codes = a_codes; p.a_scale = a_scale; p.a_zp = a_zp;
-    p.w_codes = L->codes; p.levels = L->levels; p.wsum = L->wsum; p.wscale = L->wscale; p.bias = L->bias;
+    p.a_scale = a_scale; p.a_zp = a_zp;
+    p.levels = L->levels; p.wsum = L->wsum; p.wscale = L->wscale; p.bias = L->bias;
     p.Y = Y; p.ldy = ldy; p.M = M; p.N = L->N; p.K = L->K; p.G = L->group; p.y_dtype = (int)dt;
     p.status = lrq_status_word();
-    const int tiles = ((M + BM - 1) / BM) * ((L->N + BN - 1) / BN);
-    const int grid = tiles < sms ? tiles : sms;
-    const int ab = L->act.a_bits;
-    if (ab == 8 && L->w_bits == 4) return launch<8, 4>(p, grid, st);
-    if (ab == 8) return launch<8, 3>(p, grid, st);
-    if (ab == 4 && L->w_bits == 4) return launch<4, 4>(p, grid, st);
-    return launch<4, 3>(p, grid, st);
+    // code matrices as byte tensors: a tile is 128 rows by one k-block of codes
+    const uint64_t a_row = (uint64_t)L->K * ab / 8, w_row = (uint64_t)L->K / 2;
+    CUtensorMap tmA, tmW;
+    if (!lrq_tma::make_map_2d(&tmA, a_codes, 1, (uint64_t)M, a_row, a_row, BK * ab / 8, BM_CTA, false)) return LRQ_ERR_CUDA;
+    if (!lrq_tma::make_map_2d(&tmW, L->codes, 1, (uint64_t)L->N, w_row, w_row, BK / 2, BN_CTA, false)) return LRQ_ERR_CUDA;
+    const int tiles = ((M + 2 * BM_CTA - 1) / (2 * BM_CTA)) * ((L->N + BN - 1) / BN);
+    if (ab == 8 && L->w_bits == 4) return launch<8, 4>(p, tmA, tmW, tiles, st);
+    if (ab == 8) return launch<8, 3>(p, tmA, tmW, tiles, st);
+    if (ab == 4 && L->w_bits == 4) return launch<4, 4>(p, tmA, tmW, tiles, st);
+    return launch<4, 3>(p, tmA, tmW, tiles, st);
 }

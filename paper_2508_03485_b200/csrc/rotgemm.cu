@@ -11,7 +11,7 @@
 // CTA records a code in the status word, waits (bounded) for its TMA loads in flight and unwinds.
 #include "lrq_internal.cuh"
 #include "tc_ptx.cuh"
-#include <cuda.h>
+#include "tma_host.cuh"
 
 namespace {
 using namespace lrq_tc;
@@ -214,39 +214,6 @@ rotgemm_simple_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ld
     }
 }
 
-// cuTensorMapEncodeTiled, fetched from the driver at first use (the library does not link libcuda).
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess) {
-            (void)cudaGetLastError();
-            p = nullptr;
-        }
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// bf16 matrix [rows, cols] with `ld` elements between rows; box = box_cols x box_rows, 128-byte swizzle.
-bool make_map_bf16(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_cols,
-                   uint32_t box_rows) {
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {ld * 2};
-    const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y, cudaStream_t st) {
@@ -254,8 +221,8 @@ lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void*
     const bool tc_ok = (K % 8) == 0 && (ldx % 8) == 0 && lrq_aligned(X, 16) && lrq_aligned(R, 16) && lrq_aligned(Y, 16);
     if (tc_ok) {
         CUtensorMap tmX, tmR;
-        if (!make_map_bf16(&tmX, X, (uint64_t)M, (uint64_t)K, (uint64_t)ldx, BK, BM)) return LRQ_ERR_CUDA;
-        if (!make_map_bf16(&tmR, R, (uint64_t)K, (uint64_t)K, (uint64_t)K, 64, BK)) return LRQ_ERR_CUDA;
+        if (!lrq_tma::make_map_2d(&tmX, X, 2, (uint64_t)M, (uint64_t)K, (uint64_t)ldx, BK, BM, true)) return LRQ_ERR_CUDA;
+        if (!lrq_tma::make_map_2d(&tmR, R, 2, (uint64_t)K, (uint64_t)K, (uint64_t)K, 64, BK, true)) return LRQ_ERR_CUDA;
         static bool configured = false;
         if (!configured) {
             LRQ_CUDA_TRY(cudaFuncSetAttribute(rotgemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
