@@ -18,6 +18,8 @@
 //   warps 2-9    decode TLQ weight codes through the row's level table (held in registers as two byte
 //                planes, looked up with byte permutes) into the bf16 B stage
 //   warps 10-13  expand activation codes into the bf16 A stage
+//                (the decode warps work as two groups on alternate k-blocks: fewer, longer steps per warp,
+//                and one group's barrier latencies hide behind the other's arithmetic)
 //   warps 14-17  epilogue: tcgen05.ld the finished accumulator, scale, store
 // The bf16 stages use the canonical K-major 128-byte-swizzled UMMA layout; they are written with
 // ordinary shared stores, published to the async proxy with fence.proxy.async and handed to the MMA
@@ -43,20 +45,20 @@ constexpr int BN = 256;                      // output channels per tile
 constexpr int BN_CTA = 128;                  // weight rows decoded per CTA
 constexpr int BK = 64;
 constexpr int STAGES = 4;                    // bf16 operand stages
-constexpr int CSTAGES = 4;                   // packed-code stages
+constexpr int CSTAGES = 6;                   // packed-code stages (small, so the TMA runs well ahead of the decode)
 constexpr int A_STAGE_BYTES = BM_CTA * BK * 2;      // 16 KB
 constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;      // 16 KB
 constexpr int AC_STAGE_BYTES = BM_CTA * BK;         // room for 8-bit codes (4-bit codes use half)
 constexpr int WC_STAGE_BYTES = BN_CTA * BK / 2;     // 4 KB
 constexpr int TMA_WARP = 0, MMA_WARP = 1, B_WARP0 = 2, NUM_B_WARPS = 8, A_WARP0 = 10, NUM_A_WARPS = 4;
 constexpr int EPI_WARP0 = 14, NUM_EPI_WARPS = 4;
-constexpr int NUM_DEC_WARPS = NUM_A_WARPS + NUM_B_WARPS;
+constexpr int GROUP_WARPS = (NUM_A_WARPS + NUM_B_WARPS) / 2;   // decode warps that fill one stage (two groups alternate)
 constexpr int NUM_THREADS = (EPI_WARP0 + NUM_EPI_WARPS) * 32;      // 576
 constexpr int TMEM_COLS = 512;
 
 struct __align__(8) SharedCtl {
     uint64_t cfull[CSTAGES];      // code stage filled by TMA                       (local)
-    uint64_t cempty[CSTAGES];     // code stage read by every decode warp           (local)
+    uint64_t cempty[CSTAGES];     // code stage read by the group that decodes it   (local)
     uint64_t full[STAGES];        // bf16 stage written: own decode warps (+ the peer's relay, even CTA)
     uint64_t empty[STAGES];       // bf16 stage consumed by the MMAs                (each CTA, multicast commit)
     uint64_t tmem_full[2];        // accumulator complete                           (each CTA, multicast commit)
@@ -191,10 +193,10 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
     if (threadIdx.x == 0) {
         for (int s = 0; s < CSTAGES; ++s) {
             mbar_init(smem_u32(&ctl->cfull[s]), 1);
-            mbar_init(smem_u32(&ctl->cempty[s]), NUM_DEC_WARPS);
+            mbar_init(smem_u32(&ctl->cempty[s]), GROUP_WARPS);
         }
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), rank == 0 ? NUM_DEC_WARPS + 1 : NUM_DEC_WARPS);
+            mbar_init(smem_u32(&ctl->full[s]), rank == 0 ? GROUP_WARPS + 1 : GROUP_WARPS);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -282,97 +284,117 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         }
         __syncwarp();
     } else if (warp < A_WARP0) {
-        // =============================== B decode: 32 codes of one weight row per thread ====================
+        // =============================== B decode: one weight row (64 codes) per thread =====================
+        // The eight warps form two groups that take alternate k-blocks, so that one group's barrier
+        // latencies overlap the other's arithmetic.
         const int t = threadIdx.x - B_WARP0 * 32;                  // 0..255
-        const int row = t >> 1, c = t & 1;                         // row of the CTA's 128, half of the k-block
+        const int grp = t >> 7, row = t & 127;                     // k-block parity served, row of the CTA's 128
         const int ngrp = p.K / p.G, kb_per_grp = p.G / BK;
-        uint32_t it = 0;
-        for (int tile = pair; tile < num_tiles; tile += num_pairs) {
+        uint32_t it0 = 0;
+        bool ok = true;
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, it0 += kblocks) {
             const int n_base = (tile / tiles_m) * BN + (int)rank * BN_CTA;
             const int n = min(n_base + row, p.N - 1);               // rows past N decode a valid table; never stored
             const float4* tab = reinterpret_cast<const float4*>(p.levels + (size_t)n * ngrp * NLEV);
+            const int kb0 = (grp ^ (int)it0) & 1;
             Lut L;
             float4 raw[NLEV / 4];
+            int built = -1, fetched = kb0 / kb_per_grp;             // table index held in L / in raw
+            if (kb0 < kblocks) {
 #pragma unroll
-            for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + j);
-            bool ok = true;
-            for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                if (kb % kb_per_grp == 0) {
-                    build_lut<W_BITS>(L, raw);
-                    const int g1 = kb / kb_per_grp + 1;            // fetch the next group's table a group ahead
-                    if (g1 < ngrp) {
-#pragma unroll
-                        for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)g1 * (NLEV / 4) + j);
-                    }
+                for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)fetched * (NLEV / 4) + j);
+            }
+            for (int kb = kb0; kb < kblocks; kb += 2) {
+                const uint32_t it = it0 + kb;
+                const int gi = kb / kb_per_grp;
+                if (gi != built) {
+                    build_lut<W_BITS>(L, raw);                      // raw holds table gi (fetched one step ahead)
+                    built = gi;
                 }
-                const int cs = it % CSTAGES;
+                const int gn = (kb + 2) / kb_per_grp;               // table of this thread's next k-block
+                if (kb + 2 < kblocks && gn != fetched) {
+#pragma unroll
+                    for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)gn * (NLEV / 4) + j);
+                    fetched = gn;
+                }
+                const int s = it % STAGES, cs = it % CSTAGES;
                 ok = mbar_wait_warp(smem_u32(&ctl->cfull[cs]), (it / CSTAGES) & 1, &ctl->abort_flag, p.status, 2);
                 if (!ok) break;
-                const uint4 cw = *reinterpret_cast<const uint4*>(sWc + cs * WC_STAGE_BYTES + t * 16);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->cempty[cs]));
-                uint32_t o[16];
-                decode_w<W_BITS>(cw.x, L, o); decode_w<W_BITS>(cw.y, L, o + 4);
-                decode_w<W_BITS>(cw.z, L, o + 8); decode_w<W_BITS>(cw.w, L, o + 12);
-                const int s = it % STAGES;
+                const uint4* src = reinterpret_cast<const uint4*>(sWc + cs * WC_STAGE_BYTES + row * (BK / 2));
+                const uint4 cw2[2] = {src[0], src[1]};
                 ok = mbar_wait_warp(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 3);
                 if (!ok) break;
                 unsigned char* dst = sB + s * B_STAGE_BYTES;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) sts128(dst + swz(row, 4 * c + j), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                for (int h = 0; h < 2; ++h) {
+                    const uint4 cw = cw2[h];
+                    uint32_t o[16];
+                    decode_w<W_BITS>(cw.x, L, o); decode_w<W_BITS>(cw.y, L, o + 4);
+                    decode_w<W_BITS>(cw.z, L, o + 8); decode_w<W_BITS>(cw.w, L, o + 12);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        sts128(dst + swz(row, 4 * h + j), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&ctl->full[s]));
+                    // the code stage is handed back only here: every lane's loads from it have been consumed
+                    // by the decode above, so none can still be in flight when the TMA overwrites it
+                    mbar_arrive(smem_u32(&ctl->cempty[cs]));
+                }
             }
-            if (!ok || __any_sync(0xffffffffu, ctl->abort_flag != 0)) break;
+            if (__any_sync(0xffffffffu, ctl->abort_flag != 0)) ok = false;
         }
     } else if (warp < EPI_WARP0) {
         // =============================== A expansion: 16-byte chunks of the code stage ======================
+        // Two groups of two warps, alternate k-blocks, like the B warps.
         const int t = threadIdx.x - A_WARP0 * 32;                  // 0..127
-        constexpr int TASKS = BM_CTA * AC_ROW_BYTES / 16 / (NUM_A_WARPS * 32);   // 4 (8-bit) or 2 (4-bit)
+        const int grp = t >> 6, tl = t & 63;
         constexpr int CH_PER_ROW = AC_ROW_BYTES / 16;              // 4 or 2 code chunks per token row
-        uint32_t it = 0;
-        for (int tile = pair; tile < num_tiles; tile += num_pairs) {
-            bool ok = true;
-            for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                const int cs = it % CSTAGES;
+        constexpr int TASKS = BM_CTA * CH_PER_ROW / 64;            // chunks per thread: 8 (8-bit) or 4 (4-bit)
+        constexpr int OUT_CH = 8 / CH_PER_ROW;                     // bf16 chunks per code chunk: 2 or 4
+        uint32_t it0 = 0;
+        bool ok = true;
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, it0 += kblocks) {
+            for (int kb = (grp ^ (int)it0) & 1; kb < kblocks; kb += 2) {
+                const uint32_t it = it0 + kb;
+                const int s = it % STAGES, cs = it % CSTAGES;
                 ok = mbar_wait_warp(smem_u32(&ctl->cfull[cs]), (it / CSTAGES) & 1, &ctl->abort_flag, p.status, 6);
                 if (!ok) break;
-                uint4 cw[TASKS];
+                const uint4* src = reinterpret_cast<const uint4*>(sAc + cs * AC_STAGE_BYTES);
+                uint4 cws[TASKS];
 #pragma unroll
-                for (int i = 0; i < TASKS; ++i)
-                    cw[i] = *reinterpret_cast<const uint4*>(sAc + cs * AC_STAGE_BYTES + (i * NUM_A_WARPS * 32 + t) * 16);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->cempty[cs]));
-                uint32_t o[TASKS][A_BITS == 8 ? 8 : 16];
-#pragma unroll
-                for (int i = 0; i < TASKS; ++i) {
-                    if constexpr (A_BITS == 8) {
-                        expand_a8(cw[i].x, o[i][0], o[i][1]); expand_a8(cw[i].y, o[i][2], o[i][3]);
-                        expand_a8(cw[i].z, o[i][4], o[i][5]); expand_a8(cw[i].w, o[i][6], o[i][7]);
-                    } else {
-                        expand_a4(cw[i].x, o[i]); expand_a4(cw[i].y, o[i] + 4);
-                        expand_a4(cw[i].z, o[i] + 8); expand_a4(cw[i].w, o[i] + 12);
-                    }
-                }
-                const int s = it % STAGES;
+                for (int i = 0; i < TASKS; ++i) cws[i] = src[i * 64 + tl];   // consecutive lanes read consecutive chunks
                 ok = mbar_wait_warp(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 7);
                 if (!ok) break;
                 unsigned char* dst = sA + s * A_STAGE_BYTES;
 #pragma unroll
                 for (int i = 0; i < TASKS; ++i) {
-                    const int id = i * NUM_A_WARPS * 32 + t;
+                    const int id = i * 64 + tl;
                     const int row = id / CH_PER_ROW, cc = id % CH_PER_ROW;
-                    constexpr int OUT_CH = 8 / CH_PER_ROW;         // bf16 chunks per code chunk: 2 or 4
+                    const uint4 cw = cws[i];
+                    uint32_t o[4 * OUT_CH];
+                    if constexpr (A_BITS == 8) {
+                        expand_a8(cw.x, o[0], o[1]); expand_a8(cw.y, o[2], o[3]);
+                        expand_a8(cw.z, o[4], o[5]); expand_a8(cw.w, o[6], o[7]);
+                    } else {
+                        expand_a4(cw.x, o); expand_a4(cw.y, o + 4); expand_a4(cw.z, o + 8); expand_a4(cw.w, o + 12);
+                    }
 #pragma unroll
                     for (int j = 0; j < OUT_CH; ++j)
-                        sts128(dst + swz(row, OUT_CH * cc + j), o[i][4 * j], o[i][4 * j + 1], o[i][4 * j + 2], o[i][4 * j + 3]);
+                        sts128(dst + swz(row, OUT_CH * cc + j), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&ctl->full[s]));
+                    // the code stage is handed back only here: every lane's loads from it have been consumed
+                    // by the decode above, so none can still be in flight when the TMA overwrites it
+                    mbar_arrive(smem_u32(&ctl->cempty[cs]));
+                }
             }
-            if (!ok || __any_sync(0xffffffffu, ctl->abort_flag != 0)) break;
+            if (__any_sync(0xffffffffu, ctl->abort_flag != 0)) ok = false;
         }
     } else {
         // =============================== epilogue: TMEM -> registers -> global ===============================

@@ -6,8 +6,13 @@
 
 namespace lrq_tc {
 
-// A spinning wait gives up after this many polls; the kernel then records a code and unwinds.
+// A wait gives up after this many SM clock cycles (a second or two); the kernel then records a code and
+// unwinds.  kWaitLimit bounds the polls of the drain loops that run after such an abort.
+constexpr long long kWaitCycles = 3000000000ll;
 constexpr uint32_t kWaitLimit = 1u << 22;
+// Each poll lets the hardware suspend the thread for up to this many nanoseconds while the phase is
+// pending, so that waiting warps do not compete for issue slots with the working ones.
+constexpr uint32_t kSuspendHintNs = 20000;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -33,9 +38,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
         "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok != 0;
 }
 // try_wait with cluster-scope acquire: pairs with arrivals made by another CTA of the cluster.
@@ -43,34 +48,39 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     uint32_t ok;
     asm volatile(
         "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n"
         "selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok != 0;
 }
 
 // Bounded wait.  Returns false (after raising *abort_flag and recording `code` in *status) when the
 // phase never completed, or as soon as another thread of the CTA has raised the flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    do {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-    }
+    } while (clock64() - t0 < kWaitCycles);
     *abort_flag = 1;
     if (status) atomicCAS(status, 0, code);
     return false;
 }
-// The same for a whole warp: every lane waits and all lanes get the same answer, so that warp-level
-// synchronisation after the wait stays convergent when a wait expires.
+// The same for a whole (converged) warp.  Every lane waits on the barrier itself (a lane that has not
+// observed the phase has no ordering against the asynchronous writes it guards), then the lanes agree
+// on one answer, so that warp-level synchronisation after the wait stays convergent when a wait expires.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
     const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
     return __all_sync(0xffffffffu, ok);
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    do {
         if (mbar_try_wait_cluster(bar, parity)) return true;
         if (*abort_flag) return false;
-    }
+    } while (clock64() - t0 < kWaitCycles);
     *abort_flag = 1;
     if (status) atomicCAS(status, 0, code);
     return false;
