@@ -23,8 +23,8 @@
 //   warps 14-17  epilogue: tcgen05.ld the finished accumulator, scale, store
 // The bf16 stages use the canonical K-major 128-byte-swizzled UMMA layout; they are written with
 // ordinary shared stores, published to the async proxy with fence.proxy.async and handed to the MMA
-// thread of the even CTA through an mbarrier there (in the odd CTA the decode warps arrive on a local
-// barrier and one relay thread forwards each completed stage with a single cluster-scope arrival).  Stage release and
+// thread of the even CTA through an mbarrier there (the odd CTA's warps arrive on it remotely, with
+// CTA-scope release: their data already sits, proxy-fenced, in their own shared memory by then).  Stage release and
 // accumulator completion come back to both CTAs through multicast tcgen05.commit.  The accumulator is
 // double-buffered in TMEM (2 x 256 columns) so that the epilogue of one tile overlaps the main loop of
 // the next.  Every wait is bounded: when one expires the CTA records a code in the status word, stops
@@ -59,7 +59,7 @@ constexpr int TMEM_COLS = 512;
 struct __align__(8) SharedCtl {
     uint64_t cfull[CSTAGES];      // code stage filled by TMA                       (local)
     uint64_t cempty[CSTAGES];     // code stage read by the group that decodes it   (local)
-    uint64_t full[STAGES];        // bf16 stage written: own decode warps (+ the peer's relay, even CTA)
+    uint64_t full[STAGES];        // bf16 stage written by the decode warps of both CTAs (used in the even CTA)
     uint64_t empty[STAGES];       // bf16 stage consumed by the MMAs                (each CTA, multicast commit)
     uint64_t tmem_full[2];        // accumulator complete                           (each CTA, multicast commit)
     uint64_t tmem_empty[2];       // accumulator drained by both CTAs' epilogues    (used in the even CTA)
@@ -196,7 +196,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             mbar_init(smem_u32(&ctl->cempty[s]), GROUP_WARPS);
         }
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), rank == 0 ? GROUP_WARPS + 1 : GROUP_WARPS);
+            mbar_init(smem_u32(&ctl->full[s]), 2 * GROUP_WARPS);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -268,19 +268,6 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                 }
                 if (ok) tc_commit_pair(smem_u32(&ctl->tmem_full[buf]), 3);   // accumulator complete, both halves
             }
-        } else if (rank == 1 && lane == 0) {
-            // relay: once this CTA's decode warps have all published a stage, tell the even CTA with one
-            // cluster-scope release (the decode warps themselves only pay for CTA-scope arrivals)
-            uint32_t it = 0;
-            bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    ok = mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, p.status, 9);
-                    if (!ok) break;
-                    mbar_arrive_cluster(smem_u32(&ctl->full[s]), 0);
-                }
-            }
         }
         __syncwarp();
     } else if (warp < A_WARP0) {
@@ -338,7 +325,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(smem_u32(&ctl->full[s]));
+                    mbar_arrive_cluster_light(smem_u32(&ctl->full[s]), 0);      // the even CTA's barrier
                     // the code stage is handed back only here: every lane's loads from it have been consumed
                     // by the decode above, so none can still be in flight when the TMA overwrites it
                     mbar_arrive(smem_u32(&ctl->cempty[cs]));
@@ -388,7 +375,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(smem_u32(&ctl->full[s]));
+                    mbar_arrive_cluster_light(smem_u32(&ctl->full[s]), 0);      // the even CTA's barrier
                     // the code stage is handed back only here: every lane's loads from it have been consumed
                     // by the decode above, so none can still be in flight when the TMA overwrites it
                     mbar_arrive(smem_u32(&ctl->cempty[cs]));

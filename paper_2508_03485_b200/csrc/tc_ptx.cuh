@@ -34,6 +34,16 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar, uint32_t cta_r
         "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n}"
         ::"r"(bar), "r"(cta_rank) : "memory");
 }
+// The same with the default (CTA-scope release) ordering.  A cluster-scope release costs a memory barrier
+// of a thousand cycles or more on this part; this form is enough when what the arrival publishes already
+// sits in this CTA's shared memory, made visible to the async proxy by fence.proxy.async, before it is sent.
+__device__ __forceinline__ void mbar_arrive_cluster_light(uint32_t bar, uint32_t cta_rank) {
+    asm volatile(
+        "{\n.reg .b32 ra;\n"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n}"
+        ::"r"(bar), "r"(cta_rank) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
