@@ -6,6 +6,7 @@
 // memory.  The 1/sqrt(B) normalisation is never applied to the elements: it is folded into the
 // per-token scale, since rint(y/s) is invariant under a common factor of y and s.
 #include "lrq_internal.cuh"
+#include <climits>
 
 namespace {
 
@@ -150,21 +151,54 @@ rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log
 
 
 // ------------------------------------------------------------------------------------------------
-// Fast kernel.  A thread owns 32 consecutive elements of one token (four 128-bit loads in flight):
-// index bits 0-4 of the transform are butterflies between its own registers, bits 5-9 are
-// butterflies with the lane whose index differs in one bit (one shuffle and one fused
-// multiply-add per element and stage), bits 10-11 (B = 2048, 4096) go through shared memory.
-// A CTA holds T whole tokens (T * K/32 threads, a multiple of 32); the token's extremes are reduced
-// through shared memory, then every thread quantizes and packs its own 32 values from registers:
-// 32 bytes (8-bit codes) or 16 bytes (4-bit codes) per thread, contiguous across the warp.
+// Fast kernel.  A thread owns 32 consecutive elements of one token (four 128-bit loads in flight,
+// the next token group's loads issued before the current group's arithmetic): index bits 0-4 of the
+// transform are butterflies between its own registers, bits 5-9 are butterflies with the lane whose
+// index differs in one bit (two shuffles and one packed fused multiply-add per element pair and
+// stage), bits 10-11 (B = 2048, 4096) go through shared memory.  All fp32 arithmetic on element
+// pairs uses the packed two-wide instructions (add/sub/fma.f32x2): one issue slot per two elements.
+// A CTA holds T whole tokens (T * K/32 threads, a multiple of 32) and walks over token groups with
+// a grid stride; the token's extremes are reduced through shared memory, then every thread
+// quantizes and packs its own 32 values from registers: 32 bytes (8-bit codes) or 16 bytes (4-bit
+// codes) per thread, contiguous across the warp.
 // ------------------------------------------------------------------------------------------------
 constexpr int EPT = 32;
+typedef unsigned long long f32x2;      // two fp32 values in one 64-bit register pair
+
+__device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ void unpack2(f32x2 r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+__device__ __forceinline__ float min3(float a, float b, float c) { float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
+__device__ __forceinline__ float max3(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
+
+// Order-preserving map between fp32 and int32 (and back), so that integer min/max reductions serve floats.
+__device__ __forceinline__ int ordered_int(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
+__device__ __forceinline__ float ordered_float(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
     uint4 r;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
+}
+
+// A thread's 64 input bytes.  WIDE: two 256-bit loads, so that every lane reads whole 32-byte sectors (with
+// 128-bit loads at a 64-byte lane stride each sector would be requested twice); needs 32-byte aligned rows.
+template <bool WIDE>
+__device__ __forceinline__ void load_raw(const __nv_bfloat16* p, uint4* raw) {
+    if (WIDE) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+            asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(raw[2 * i].x), "=r"(raw[2 * i].y), "=r"(raw[2 * i].z), "=r"(raw[2 * i].w),
+                           "=r"(raw[2 * i + 1].x), "=r"(raw[2 * i + 1].y), "=r"(raw[2 * i + 1].z), "=r"(raw[2 * i + 1].w)
+                         : "l"(p + 16 * i));
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) raw[i] = ldg_stream(reinterpret_cast<const uint4*>(p) + i);
+    }
 }
 
 __device__ __forceinline__ uint32_t pack_u8x4(int q0, int q1, int q2, int q3) {
@@ -182,110 +216,191 @@ __device__ __forceinline__ uint32_t pack_u4x8(const int* q) {
     return t;
 }
 
-template <int LOG2B, int A_BITS>
-__global__ void __launch_bounds__(512)
-rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, int mode, int tok_per_cta,
+// The same parameters for the fast kernel, where every warp works them out: one fp64 reciprocal refined
+// from the fp32 approximation (two Newton steps, relative error below 1e-14) instead of fp64 divisions.
+__device__ __forceinline__ TokenQ token_params_fast(float mn, float mx, int a_bits, int mode, double nrm,
+                                                    float* scale_out, int32_t* zp_out) {
+    const bool asym = mode == LRQ_ACT_ASYM;
+    const double qsteps = asym ? (double)((1 << a_bits) - 1) : (double)((1 << (a_bits - 1)) - 1);
+    const double range = asym ? (double)mx - (double)mn : (double)fmaxf(fabsf(mn), fabsf(mx));
+    const float r0 = __frcp_rn((float)range);
+    double s, inv;
+    if (range > 0.0 && r0 > 0.f && r0 < 3.0e38f) {
+        double r = (double)r0;
+        r = fma(r, fma(-range, r, 1.0), r);
+        r = fma(r, fma(-range, r, 1.0), r);
+        inv = qsteps * r;
+        s = range * (1.0 / qsteps);
+    } else if (range > 0.0) {      // outside fp32's reciprocal range: plain division
+        s = range / qsteps;
+        inv = 1.0 / s;
+    } else {                       // empty range: unit step in the normalised domain
+        s = 1.0 / nrm;
+        inv = nrm;
+    }
+    const double z = asym ? rint((double)mn * inv) : -(double)(1 << (a_bits - 1));
+    *scale_out = (float)(s * nrm);
+    *zp_out = (int32_t)z;
+    TokenQ t;
+    t.inv = (float)inv;
+    t.negz = (float)(-z);
+    return t;
+}
+
+template <int LOG2B, int A_BITS, int MAX_THREADS, int MIN_CTAS, bool WIDE>
+__global__ void __launch_bounds__(MAX_THREADS, MIN_CTAS)
+rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, int mode, int tok_per_cta, int num_groups,
                  uint8_t* __restrict__ codes, float* __restrict__ scale, int32_t* __restrict__ zp) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    constexpr int NP = EPT / 2;                      // element pairs per thread
     const int tpt = K / EPT;                         // threads per token
     const int tid = threadIdx.x, lane = tid & 31;
     const int tl = tid / tpt, j = tid - tl * tpt;    // token within the CTA, thread within the token
-    const int m = blockIdx.x * tok_per_cta + tl;
-    const bool live = m < M;
+    int* ext = reinterpret_cast<int*>(smem_raw);     // [3][tok_per_cta][2] token extremes (ordered ints), rotating
+    // lanes of this warp that belong to the same token, and the lowest of them
+    const unsigned seg_mask = __match_any_sync(0xffffffffu, tl);
+    const int seg_lane = __ffs(seg_mask) - 1;
+    const bool seg_leader = lane == seg_lane;
+    for (int i = tid; i < 3 * 2 * tok_per_cta; i += blockDim.x) ext[i] = (i & 1) ? INT_MIN : INT_MAX;
+    __syncthreads();
 
-    float v[EPT];
-    if (live) {
-        const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)m * ldx + (size_t)j * EPT);
-        uint4 r[4];
+    uint4 raw[4];
+    {
+        const int m = blockIdx.x * tok_per_cta + tl;
+        if (m < M) {
+            load_raw<WIDE>(X + (size_t)m * ldx + (size_t)j * EPT, raw);
+        } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) r[i] = ldg_stream(src + i);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) unpack_bf16x8(r[i], v + 8 * i);
-    } else {
-#pragma unroll
-        for (int i = 0; i < EPT; ++i) v[i] = 0.f;
-    }
-    // index bits 0..4: registers
-#pragma unroll
-    for (int h = 1; h < EPT && h < (1 << LOG2B); h <<= 1)
-#pragma unroll
-        for (int i = 0; i < EPT; ++i)
-            if (!(i & h)) { const float a = v[i], b = v[i | h]; v[i] = a + b; v[i | h] = a - b; }
-    // index bits 5..9: partner lanes
-#pragma unroll
-    for (int b = 5; b < LOG2B && b < 10; ++b) {
-        const int lm = 1 << (b - 5);
-        const float sgn = (lane & lm) ? -1.f : 1.f;
-#pragma unroll
-        for (int i = 0; i < EPT; ++i) {
-            const float o = __shfl_xor_sync(0xffffffffu, v[i], lm);
-            v[i] = fmaf(v[i], sgn, o);               // low lane: own + other, high lane: other - own
+            for (int i = 0; i < 4; ++i) raw[i] = make_uint4(0, 0, 0, 0);
         }
     }
-    // index bits 10..11: partner warps, through shared memory (chunk index swizzled by the lane)
-    float* red = reinterpret_cast<float*>(smem_raw);                 // [3][nthreads]
-    TokenQ* tqs = reinterpret_cast<TokenQ*>(red + 3 * blockDim.x);   // [tok_per_cta]
-    if (LOG2B > 10) {
-        float4* xb = reinterpret_cast<float4*>(tqs + tok_per_cta + 1);
-        xb = reinterpret_cast<float4*>((reinterpret_cast<uintptr_t>(xb) + 15) & ~uintptr_t(15));
+    int it = 0;
+    for (int g = blockIdx.x; g < num_groups; g += gridDim.x, ++it) {
+        const int m = g * tok_per_cta + tl;
+        const bool live = m < M;
+        // bf16 -> fp32, two elements per word
+        f32x2 P[NP];
 #pragma unroll
-        for (int b = 10; b < LOG2B; ++b) {
-            const int tm = 1 << (b - 5);
-            __syncthreads();
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                xb[tid * 8 + (c ^ (lane & 7))] = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
-            __syncthreads();
-            const int pt = tid ^ tm;
-            const float sgn = (tid & tm) ? -1.f : 1.f;
+            for (int c = 0; c < 4; ++c)
+                P[4 * i + c] = pack2(__uint_as_float(w[c] << 16), __uint_as_float(w[c] & 0xffff0000u));
+        }
+        // the next group's loads fly while this group is transformed
+        {
+            const int mn = (g + (int)gridDim.x) * tok_per_cta + tl;
+            if (g + (int)gridDim.x < num_groups && mn < M) {
+                load_raw<WIDE>(X + (size_t)mn * ldx + (size_t)j * EPT, raw);
+            } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const float4 o = xb[pt * 8 + (c ^ (lane & 7))];
-                v[4 * c] = fmaf(v[4 * c], sgn, o.x); v[4 * c + 1] = fmaf(v[4 * c + 1], sgn, o.y);
-                v[4 * c + 2] = fmaf(v[4 * c + 2], sgn, o.z); v[4 * c + 3] = fmaf(v[4 * c + 3], sgn, o.w);
+                for (int i = 0; i < 4; ++i) raw[i] = make_uint4(0, 0, 0, 0);
             }
         }
-    }
-    // extremes of the thread's values, then of the token
-    float mn = v[0], mx = v[0];
+        // index bit 0: the two halves of a pair
 #pragma unroll
-    for (int i = 1; i < EPT; ++i) { mn = fminf(mn, v[i]); mx = fmaxf(mx, v[i]); }
-    __syncthreads();
-    red[tid] = mn; red[blockDim.x + tid] = mx;
-    __syncthreads();
-    const int warp = tid >> 5, nwarp = blockDim.x >> 5;
-    for (int t = warp; t < tok_per_cta; t += nwarp) {
-        float a = INFINITY, b = -INFINITY;
-        for (int i = lane; i < tpt; i += 32) { a = fminf(a, red[t * tpt + i]); b = fmaxf(b, red[blockDim.x + t * tpt + i]); }
+        for (int i = 0; i < NP; ++i) { float a, b; unpack2(P[i], a, b); P[i] = pack2(a + b, a - b); }
+        // index bits 1..4: between pairs
 #pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            a = fminf(a, __shfl_xor_sync(0xffffffffu, a, o));
-            b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, o));
+        for (int h = 1; h < NP && (2 * h) < (1 << LOG2B); h <<= 1)
+#pragma unroll
+            for (int i = 0; i < NP; ++i)
+                if (!(i & h)) { const f32x2 a = P[i], b = P[i | h]; P[i] = add2(a, b); P[i | h] = sub2(a, b); }
+        // index bits 5..9: partner lanes
+#pragma unroll
+        for (int b = 5; b < LOG2B && b < 10; ++b) {
+            const int lm = 1 << (b - 5);
+            const float sg = (lane & lm) ? -1.f : 1.f;
+            const f32x2 S = pack2(sg, sg);
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                float x, y;
+                unpack2(P[i], x, y);
+                const float ox = __shfl_xor_sync(0xffffffffu, x, lm), oy = __shfl_xor_sync(0xffffffffu, y, lm);
+                P[i] = fma2(P[i], S, pack2(ox, oy));     // low lane: own + other, high lane: other - own
+            }
         }
-        const int mt = blockIdx.x * tok_per_cta + t;
-        if (lane == 0 && mt < M)
-            tqs[t] = token_params(a, b, fmaxf(fabsf(a), fabsf(b)), A_BITS, mode, 1.0 / sqrt((double)(1 << LOG2B)),
-                                  scale + mt, zp + mt);
-    }
-    __syncthreads();
-    if (!live) return;
-    const TokenQ t = tqs[tl];
-    int q[EPT];
+        // index bits 10..11: partner warps, through shared memory (chunk index swizzled by the lane)
+        if (LOG2B > 10) {
+            ulonglong2* xb = reinterpret_cast<ulonglong2*>(ext + 3 * 2 * tok_per_cta);
+            xb = reinterpret_cast<ulonglong2*>((reinterpret_cast<uintptr_t>(xb) + 15) & ~uintptr_t(15));
 #pragma unroll
-    for (int i = 0; i < EPT; ++i) q[i] = __float2int_rn(fmaf(v[i], t.inv, t.negz));
-    if (A_BITS == 8) {
-        uint4* dst = reinterpret_cast<uint4*>(codes + (size_t)m * K + (size_t)j * EPT);
-        uint32_t w[8];
+            for (int b = 10; b < LOG2B; ++b) {
+                const int tm = 1 << (b - 5);
+                __syncthreads();
 #pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = pack_u8x4(q[4 * i], q[4 * i + 1], q[4 * i + 2], q[4 * i + 3]);
-        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-    } else {
-        uint4* dst = reinterpret_cast<uint4*>(codes + (((size_t)m * K + (size_t)j * EPT) >> 1));
-        uint32_t w[4];
+                for (int c = 0; c < 8; ++c) xb[tid * 8 + (c ^ (lane & 7))] = make_ulonglong2(P[2 * c], P[2 * c + 1]);
+                __syncthreads();
+                const int pt = tid ^ tm;
+                const float sg = (tid & tm) ? -1.f : 1.f;
+                const f32x2 S = pack2(sg, sg);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) w[i] = pack_u4x8(q + 8 * i);
-        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                for (int c = 0; c < 8; ++c) {
+                    const ulonglong2 o = xb[pt * 8 + (c ^ (lane & 7))];
+                    P[2 * c] = fma2(P[2 * c], S, o.x);
+                    P[2 * c + 1] = fma2(P[2 * c + 1], S, o.y);
+                }
+            }
+        }
+        // extremes of the thread's values, of the token's lanes in this warp (one redux each on order-preserving
+        // integer images), then of the token: one shared-memory atomic per warp and token, one CTA barrier
+        float mn, mx;
+        unpack2(P[0], mn, mx);
+        { const float t0 = fminf(mn, mx); mx = fmaxf(mn, mx); mn = t0; }
+#pragma unroll
+        for (int i = 1; i < NP; ++i) { float x, y; unpack2(P[i], x, y); mn = min3(mn, x, y); mx = max3(mx, x, y); }
+        int* slot = ext + (it % 3) * 2 * tok_per_cta + 2 * tl;
+        {
+            const int imn = __reduce_min_sync(seg_mask, ordered_int(mn)), imx = __reduce_max_sync(seg_mask, ordered_int(mx));
+            if (seg_leader) { atomicMin(slot, imn); atomicMax(slot + 1, imx); }
+        }
+        __syncthreads();
+        // every warp works out its token's step and zero-point itself (one lane, fp64): no second barrier
+        TokenQ t;
+        {
+            float sc = 0.f; int z = 0;
+            t.inv = 0.f; t.negz = 0.f;
+            if (seg_leader) {
+                const float a = ordered_float(slot[0]), b = ordered_float(slot[1]);
+                t = token_params_fast(a, b, A_BITS, mode, 1.0 / sqrt((double)(1 << LOG2B)), &sc, &z);
+                if (j == 0 && live) { scale[m] = sc; zp[m] = z; }
+            }
+            t.inv = __shfl_sync(seg_mask, t.inv, seg_lane);
+            t.negz = __shfl_sync(seg_mask, t.negz, seg_lane);
+        }
+        // the slots used two groups from now are reset here: their last readers passed the barrier above, and
+        // their next writers come after the next barrier
+        if (tid < 2 * tok_per_cta) ext[((it + 2) % 3) * 2 * tok_per_cta + tid] = (tid & 1) ? INT_MIN : INT_MAX;
+        if (live) {
+            const f32x2 INV = pack2(t.inv, t.inv), NEGZ = pack2(t.negz, t.negz);
+            int q[EPT];
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                float x, y;
+                unpack2(fma2(P[i], INV, NEGZ), x, y);
+                q[2 * i] = __float2int_rn(x); q[2 * i + 1] = __float2int_rn(y);
+            }
+            if (A_BITS == 8) {
+                uint4* dst = reinterpret_cast<uint4*>(codes + (size_t)m * K + (size_t)j * EPT);
+                uint32_t w[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) w[i] = pack_u8x4(q[4 * i], q[4 * i + 1], q[4 * i + 2], q[4 * i + 3]);
+                if (WIDE) {
+                    asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                 :: "l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                                 : "memory");
+                } else {
+                    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+            } else {
+                uint4* dst = reinterpret_cast<uint4*>(codes + (((size_t)m * K + (size_t)j * EPT) >> 1));
+                uint32_t w[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) w[i] = pack_u4x8(q + 8 * i);
+                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
     }
 }
 
@@ -315,11 +430,29 @@ static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits,
     while (T * tpt < 256 && (T + T0) * tpt <= 512) T += T0;
     const int threads = T * tpt;
     if (threads > 512) return LRQ_ERR_UNSUPPORTED;
-    size_t smem = 3 * sizeof(float) * threads + sizeof(TokenQ) * (T + 1) + 16;
+    size_t smem = 3 * 2 * sizeof(int) * T + 16;
     if (LOG2B > 10) smem += (size_t)threads * EPT * sizeof(float);
-    auto kern = a_bits == 8 ? rotq_fast_kernel<LOG2B, 8> : rotq_fast_kernel<LOG2B, 4>;
+    // register budget by CTA size: three CTAs of up to 288 threads, two of up to 384, else one
+    typedef void (*Kern)(const __nv_bfloat16*, int, int, long, int, int, int, uint8_t*, float*, int32_t*);
+    // 256-bit accesses when every thread's 64 input bytes and 32 code bytes start on 32-byte boundaries
+    const bool wide = lrq_aligned(X, 32) && (ldx % 16) == 0 && lrq_aligned(codes, 32);
+    Kern kern;
+#define LRQ_PICK(NT, NB) (wide ? (a_bits == 8 ? rotq_fast_kernel<LOG2B, 8, NT, NB, true> : rotq_fast_kernel<LOG2B, 4, NT, NB, true>) \
+                               : (a_bits == 8 ? rotq_fast_kernel<LOG2B, 8, NT, NB, false> : rotq_fast_kernel<LOG2B, 4, NT, NB, false>))
+    if (threads <= 288) kern = LRQ_PICK(288, 3);
+    else if (threads <= 384) kern = LRQ_PICK(384, 2);
+    else kern = LRQ_PICK(512, 1);
+#undef LRQ_PICK
     if (smem > 40 * 1024) LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<(M + T - 1) / T, threads, smem, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx, mode, T, codes, scale, zp);
+    // persistent grid: as many CTAs as stay resident, each walking over token groups with a grid stride
+    int dev = 0, sms = 0, per_sm = 0;
+    LRQ_CUDA_TRY(cudaGetDevice(&dev));
+    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    LRQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem));
+    if (per_sm < 1) return LRQ_ERR_UNSUPPORTED;
+    const int groups = (M + T - 1) / T;
+    const int grid = groups < sms * per_sm ? groups : sms * per_sm;
+    kern<<<grid, threads, smem, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx, mode, T, groups, codes, scale, zp);
     LRQ_CUDA_TRY(cudaGetLastError());
     return LRQ_OK;
 }
