@@ -56,7 +56,7 @@ constexpr int GROUP_WARPS = (NUM_A_WARPS + NUM_B_WARPS) / 2;   // decode warps t
 constexpr int NUM_THREADS = (EPI_WARP0 + NUM_EPI_WARPS) * 32;      // 576
 constexpr int TMEM_COLS = 512;
 
-struct __align__(8) SharedCtl {
+struct __align__(16) SharedCtl {
     uint64_t cfull[CSTAGES];      // code stage filled by TMA                       (local)
     uint64_t cempty[CSTAGES];     // code stage read by the group that decodes it   (local)
     uint64_t full[STAGES];        // bf16 stage written by the decode warps of both CTAs (used in the even CTA)
@@ -65,7 +65,7 @@ struct __align__(8) SharedCtl {
     uint64_t tmem_empty[2];       // accumulator drained by both CTAs' epilogues    (used in the even CTA)
     uint32_t tmem_base;
     volatile int abort_flag;
-    float col[2][3][BN];          // per TMEM buffer: wsum, wscale, bias of the tile's columns
+    alignas(16) float col[2][3][BN];   // per TMEM buffer: wsum, wscale, bias of the tile's columns (read as float4)
 };
 
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
@@ -97,13 +97,15 @@ __device__ __forceinline__ void expand_a8(uint32_t w, uint32_t& o01, uint32_t& o
     o23 = add_bf16x2((p23 & 0x007F007Fu) | 0x43004300u, (p23 & 0x00800080u) ^ 0xC380C380u);
 }
 // 4-bit: eight codes per word -> bf16 of (q - 8): 0x4300 | q is 128 + q, and 128 + q - 136 is exact.
+// The eight elements come out in the order k = 0,2, 4,6, 1,3, 5,7 within the word (one byte permute per
+// pair instead of a permute and an OR); the weight decode of 4-bit-activation layers emits the same order,
+// and a contraction does not care in which order k is summed as long as both operands agree.
 __device__ __forceinline__ void expand_a4(uint32_t w, uint32_t* o) {
     const uint32_t lo = w & 0x0F0F0F0Fu, hi = (w >> 4) & 0x0F0F0F0Fu;      // even / odd codes, one per byte
-    // bytes below 16 have a clear top bit: selector 8|k yields 0x00
-    o[0] = add_bf16x2(prmt(lo, hi, 0x8480u) | 0x43004300u, 0xC308C308u);
-    o[1] = add_bf16x2(prmt(lo, hi, 0x8581u) | 0x43004300u, 0xC308C308u);
-    o[2] = add_bf16x2(prmt(lo, hi, 0x8682u) | 0x43004300u, 0xC308C308u);
-    o[3] = add_bf16x2(prmt(lo, hi, 0x8783u) | 0x43004300u, 0xC308C308u);
+    o[0] = add_bf16x2(prmt(lo, 0x43434343u, 0x4140u), 0xC308C308u);        // codes 0, 2
+    o[1] = add_bf16x2(prmt(lo, 0x43434343u, 0x4342u), 0xC308C308u);        // codes 4, 6
+    o[2] = add_bf16x2(prmt(hi, 0x43434343u, 0x4140u), 0xC308C308u);        // codes 1, 3
+    o[3] = add_bf16x2(prmt(hi, 0x43434343u, 0x4342u), 0xC308C308u);        // codes 5, 7
 }
 
 // ---- TLQ codes -> bf16 through the row's level table ------------------------------------------------
@@ -126,9 +128,12 @@ __device__ __forceinline__ void build_lut(Lut& L, const float4* raw) {
     }
 }
 
-// eight codes (one word) -> four registers of two bf16 each, in k order
-template <int W_BITS>
+// eight codes (one word) -> four registers of two bf16 each: in k order, or (A4_ORDER) in the order
+// 0,2, 4,6, 1,3, 5,7 that the 4-bit activation expansion produces
+template <int W_BITS, bool A4_ORDER>
 __device__ __forceinline__ void decode_w(uint32_t w, const Lut& L, uint32_t* o) {
+    // loA/hiA hold codes 0-3, loB/hiB codes 4-7 (one byte each); output register = two (lo, hi) byte pairs
+    constexpr uint32_t S0 = A4_ORDER ? 0x6240u : 0x5140u, S1 = A4_ORDER ? 0x7351u : 0x7362u;
     if (W_BITS == 4) {
         const uint32_t selA = w & 0x77777777u, selB = selA >> 16;
         const uint32_t x0 = w << 4;
@@ -137,14 +142,14 @@ __device__ __forceinline__ void decode_w(uint32_t w, const Lut& L, uint32_t* o) 
         const uint32_t hiA = (prmt(L.hi[0], L.hi[1], selA) & ~mA) | (prmt(L.hi[2], L.hi[3], selA) & mA);
         const uint32_t loB = (prmt(L.lo[0], L.lo[1], selB) & ~mB) | (prmt(L.lo[2], L.lo[3], selB) & mB);
         const uint32_t hiB = (prmt(L.hi[0], L.hi[1], selB) & ~mB) | (prmt(L.hi[2], L.hi[3], selB) & mB);
-        o[0] = prmt(loA, hiA, 0x5140u); o[1] = prmt(loA, hiA, 0x7362u);
-        o[2] = prmt(loB, hiB, 0x5140u); o[3] = prmt(loB, hiB, 0x7362u);
+        if (A4_ORDER) { o[0] = prmt(loA, hiA, S0); o[1] = prmt(loB, hiB, S0); o[2] = prmt(loA, hiA, S1); o[3] = prmt(loB, hiB, S1); }
+        else { o[0] = prmt(loA, hiA, S0); o[1] = prmt(loA, hiA, S1); o[2] = prmt(loB, hiB, S0); o[3] = prmt(loB, hiB, S1); }
     } else {                                   // at most 8 table entries: one permute per plane
         const uint32_t selA = w & 0x77777777u, selB = selA >> 16;
         const uint32_t loA = prmt(L.lo[0], L.lo[1], selA), hiA = prmt(L.hi[0], L.hi[1], selA);
         const uint32_t loB = prmt(L.lo[0], L.lo[1], selB), hiB = prmt(L.hi[0], L.hi[1], selB);
-        o[0] = prmt(loA, hiA, 0x5140u); o[1] = prmt(loA, hiA, 0x7362u);
-        o[2] = prmt(loB, hiB, 0x5140u); o[3] = prmt(loB, hiB, 0x7362u);
+        if (A4_ORDER) { o[0] = prmt(loA, hiA, S0); o[1] = prmt(loB, hiB, S0); o[2] = prmt(loA, hiA, S1); o[3] = prmt(loB, hiB, S1); }
+        else { o[0] = prmt(loA, hiA, S0); o[1] = prmt(loA, hiA, S1); o[2] = prmt(loB, hiB, S0); o[3] = prmt(loB, hiB, S1); }
     }
 }
 
@@ -159,9 +164,33 @@ __device__ __forceinline__ bool bar_or_epilogue(bool pred) {
     return r != 0;
 }
 
-__device__ __forceinline__ void sts128(unsigned char* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
+// 128-bit shared-memory accesses on 32-bit shared addresses (no 64-bit pointer arithmetic in the inner loops)
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+__device__ __forceinline__ void lds128(uint32_t addr, uint4& v) {
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+}
+
+// Ring positions of a decode group.  A group serves every second k-block of the CTA's running count, so its
+// slot in the 4-deep operand ring alternates between two values and its slot in the code ring advances by two;
+// the phase bits flip when a slot index wraps.
+struct RingPos {
+    uint32_t s, ph, cs, cph;
+    __device__ explicit RingPos(int grp) : s((uint32_t)grp), ph(0), cs((uint32_t)grp), cph(0) {}
+    __device__ __forceinline__ void advance() {
+        s += 2; if (s >= (uint32_t)STAGES) { s -= STAGES; ph ^= 1; }
+        cs += 2; if (cs >= (uint32_t)CSTAGES) { cs -= CSTAGES; cph ^= 1; }
+    }
+};
+static_assert(STAGES % 2 == 0 && CSTAGES % 2 == 0, "the two decode groups own alternate ring slots");
+
+typedef unsigned long long f32x2;      // two fp32 values in one 64-bit register pair
+__device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ void unpack2(f32x2 r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
 
 struct Params {
     const float* a_scale; const int32_t* a_zp;
@@ -225,7 +254,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                 const int n_base = (tile / tiles_m) * BN + (int)rank * BN_CTA;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int cs = it % CSTAGES;
-                    ok = mbar_wait(smem_u32(&ctl->cempty[cs]), ((it / CSTAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 1);
+                    ok = mbar_wait<200>(smem_u32(&ctl->cempty[cs]), ((it / CSTAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 1);
                     if (!ok) break;
                     const uint32_t bar = smem_u32(&ctl->cfull[cs]);
                     mbar_arrive_expect_tx(bar, CODE_TX_BYTES);
@@ -250,13 +279,13 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++t) {
                 const int buf = t & 1;
-                ok = mbar_wait_cluster(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, p.status, 4);
+                ok = mbar_wait_cluster<64>(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, p.status, 4);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
-                    ok = mbar_wait_cluster(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, p.status, 5);
+                    ok = mbar_wait_cluster<32>(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, p.status, 5);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(sA + s * A_STAGE_BYTES), b_addr = smem_u32(sB + s * B_STAGE_BYTES);
@@ -273,10 +302,17 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
     } else if (warp < A_WARP0) {
         // =============================== B decode: one weight row (64 codes) per thread =====================
         // The eight warps form two groups that take alternate k-blocks, so that one group's barrier
-        // latencies overlap the other's arithmetic.
+        // latencies overlap the other's arithmetic.  A group's k-blocks are every second one of the CTA's
+        // running count, across tile boundaries too, so ring slots and phases advance by fixed steps.
         const int t = threadIdx.x - B_WARP0 * 32;                  // 0..255
         const int grp = t >> 7, row = t & 127;                     // k-block parity served, row of the CTA's 128
         const int ngrp = p.K / p.G, kb_per_grp = p.G / BK;
+        // the row's eight 16-byte chunk slots in a swizzled stage, and its 32 code bytes in a code stage
+        uint32_t off[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) off[c] = swz(row, c);
+        const uint32_t sB0 = smem_u32(sB), sWc0 = smem_u32(sWc) + (uint32_t)row * (BK / 2);
+        RingPos ring(grp);
         uint32_t it0 = 0;
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, it0 += kblocks) {
@@ -286,80 +322,97 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             const int kb0 = (grp ^ (int)it0) & 1;
             Lut L;
             float4 raw[NLEV / 4];
-            int built = -1, fetched = kb0 / kb_per_grp;             // table index held in L / in raw
+            // table index held in L / in raw, and the k-block at which the next table starts
+            int gi = kb0 / kb_per_grp, fetched = gi, next_switch = (gi + 1) * kb_per_grp;
             if (kb0 < kblocks) {
 #pragma unroll
-                for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)fetched * (NLEV / 4) + j);
+                for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)gi * (NLEV / 4) + j);
+                build_lut<W_BITS>(L, raw);
             }
             for (int kb = kb0; kb < kblocks; kb += 2) {
-                const uint32_t it = it0 + kb;
-                const int gi = kb / kb_per_grp;
-                if (gi != built) {
-                    build_lut<W_BITS>(L, raw);                      // raw holds table gi (fetched one step ahead)
-                    built = gi;
-                }
-                const int gn = (kb + 2) / kb_per_grp;               // table of this thread's next k-block
-                if (kb + 2 < kblocks && gn != fetched) {
+                if (ngrp > 1) {                                     // grouped tables: switch, and fetch one step ahead
+                    if (kb >= next_switch) {
+                        while (kb >= next_switch) { ++gi; next_switch += kb_per_grp; }
+                        if (fetched != gi) {
 #pragma unroll
-                    for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)gn * (NLEV / 4) + j);
-                    fetched = gn;
+                            for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)gi * (NLEV / 4) + j);
+                            fetched = gi;
+                        }
+                        build_lut<W_BITS>(L, raw);
+                    }
+                    if (kb + 2 >= next_switch && kb + 2 < kblocks) {
+                        int gn = gi, ns = next_switch;
+                        while (kb + 2 >= ns) { ++gn; ns += kb_per_grp; }
+                        if (gn != fetched) {
+#pragma unroll
+                            for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)gn * (NLEV / 4) + j);
+                            fetched = gn;
+                        }
+                    }
                 }
-                const int s = it % STAGES, cs = it % CSTAGES;
-                ok = mbar_wait_warp(smem_u32(&ctl->cfull[cs]), (it / CSTAGES) & 1, &ctl->abort_flag, p.status, 2);
+                ok = mbar_wait_warp<64>(smem_u32(&ctl->cfull[ring.cs]), ring.cph, &ctl->abort_flag, p.status, 2);
                 if (!ok) break;
-                const uint4* src = reinterpret_cast<const uint4*>(sWc + cs * WC_STAGE_BYTES + row * (BK / 2));
-                const uint4 cw2[2] = {src[0], src[1]};
-                ok = mbar_wait_warp(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 3);
+                uint4 cw2[2];
+                lds128(sWc0 + ring.cs * WC_STAGE_BYTES, cw2[0]);
+                lds128(sWc0 + ring.cs * WC_STAGE_BYTES + 16, cw2[1]);
+                ok = mbar_wait_warp<64>(smem_u32(&ctl->empty[ring.s]), ring.ph ^ 1, &ctl->abort_flag, p.status, 3);
                 if (!ok) break;
-                unsigned char* dst = sB + s * B_STAGE_BYTES;
+                const uint32_t dst = sB0 + ring.s * B_STAGE_BYTES;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     const uint4 cw = cw2[h];
                     uint32_t o[16];
-                    decode_w<W_BITS>(cw.x, L, o); decode_w<W_BITS>(cw.y, L, o + 4);
-                    decode_w<W_BITS>(cw.z, L, o + 8); decode_w<W_BITS>(cw.w, L, o + 12);
+                    decode_w<W_BITS, A_BITS == 4>(cw.x, L, o); decode_w<W_BITS, A_BITS == 4>(cw.y, L, o + 4);
+                    decode_w<W_BITS, A_BITS == 4>(cw.z, L, o + 8); decode_w<W_BITS, A_BITS == 4>(cw.w, L, o + 12);
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        sts128(dst + swz(row, 4 * h + j), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                        sts128(dst + off[4 * h + j], o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                 }
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_cluster_light(smem_u32(&ctl->full[s]), 0);      // the even CTA's barrier
+                    mbar_arrive_cluster_light(smem_u32(&ctl->full[ring.s]), 0);      // the even CTA's barrier
                     // the code stage is handed back only here: every lane's loads from it have been consumed
                     // by the decode above, so none can still be in flight when the TMA overwrites it
-                    mbar_arrive(smem_u32(&ctl->cempty[cs]));
+                    mbar_arrive(smem_u32(&ctl->cempty[ring.cs]));
                 }
+                ring.advance();
             }
             if (__any_sync(0xffffffffu, ctl->abort_flag != 0)) ok = false;
         }
     } else if (warp < EPI_WARP0) {
         // =============================== A expansion: 16-byte chunks of the code stage ======================
-        // Two groups of two warps, alternate k-blocks, like the B warps.
+        // Two groups of two warps, alternate k-blocks, like the B warps.  Chunk id = i * 64 + tl: consecutive
+        // lanes read consecutive chunks; the row's low three bits, hence the swizzle, do not depend on i.
         const int t = threadIdx.x - A_WARP0 * 32;                  // 0..127
         const int grp = t >> 6, tl = t & 63;
         constexpr int CH_PER_ROW = AC_ROW_BYTES / 16;              // 4 or 2 code chunks per token row
         constexpr int TASKS = BM_CTA * CH_PER_ROW / 64;            // chunks per thread: 8 (8-bit) or 4 (4-bit)
         constexpr int OUT_CH = 8 / CH_PER_ROW;                     // bf16 chunks per code chunk: 2 or 4
+        constexpr int ROWS_PER_TASK = 64 / CH_PER_ROW;             // rows between a thread's consecutive chunks
+        const int row0 = tl / CH_PER_ROW, cc = tl % CH_PER_ROW;
+        uint32_t off[OUT_CH];
+#pragma unroll
+        for (int j = 0; j < OUT_CH; ++j) off[j] = swz(row0, OUT_CH * cc + j);
+        const uint32_t sA0 = smem_u32(sA), sAc0 = smem_u32(sAc) + (uint32_t)tl * 16;
+        RingPos ring(grp);
         uint32_t it0 = 0;
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, it0 += kblocks) {
             for (int kb = (grp ^ (int)it0) & 1; kb < kblocks; kb += 2) {
-                const uint32_t it = it0 + kb;
-                const int s = it % STAGES, cs = it % CSTAGES;
-                ok = mbar_wait_warp(smem_u32(&ctl->cfull[cs]), (it / CSTAGES) & 1, &ctl->abort_flag, p.status, 6);
+                ok = mbar_wait_warp<64>(smem_u32(&ctl->cfull[ring.cs]), ring.cph, &ctl->abort_flag, p.status, 6);
                 if (!ok) break;
-                const uint4* src = reinterpret_cast<const uint4*>(sAc + cs * AC_STAGE_BYTES);
+                const uint32_t src = sAc0 + ring.cs * AC_STAGE_BYTES;
                 uint4 cws[TASKS];
 #pragma unroll
-                for (int i = 0; i < TASKS; ++i) cws[i] = src[i * 64 + tl];   // consecutive lanes read consecutive chunks
-                ok = mbar_wait_warp(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 7);
+                for (int i = 0; i < TASKS; ++i) lds128(src + i * 1024, cws[i]);
+                ok = mbar_wait_warp<64>(smem_u32(&ctl->empty[ring.s]), ring.ph ^ 1, &ctl->abort_flag, p.status, 7);
                 if (!ok) break;
-                unsigned char* dst = sA + s * A_STAGE_BYTES;
+                uint32_t dst[OUT_CH];
+#pragma unroll
+                for (int j = 0; j < OUT_CH; ++j) dst[j] = sA0 + ring.s * A_STAGE_BYTES + off[j];
 #pragma unroll
                 for (int i = 0; i < TASKS; ++i) {
-                    const int id = i * 64 + tl;
-                    const int row = id / CH_PER_ROW, cc = id % CH_PER_ROW;
                     const uint4 cw = cws[i];
                     uint32_t o[4 * OUT_CH];
                     if constexpr (A_BITS == 8) {
@@ -369,17 +422,16 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                         expand_a4(cw.x, o); expand_a4(cw.y, o + 4); expand_a4(cw.z, o + 8); expand_a4(cw.w, o + 12);
                     }
 #pragma unroll
-                    for (int j = 0; j < OUT_CH; ++j)
-                        sts128(dst + swz(row, OUT_CH * cc + j), o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                    for (int j = 0; j < OUT_CH; ++j)      // ROWS_PER_TASK rows further down: whole 1024-byte groups
+                        sts128(dst[j] + i * (ROWS_PER_TASK / 8) * 1024, o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                 }
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_cluster_light(smem_u32(&ctl->full[s]), 0);      // the even CTA's barrier
-                    // the code stage is handed back only here: every lane's loads from it have been consumed
-                    // by the decode above, so none can still be in flight when the TMA overwrites it
-                    mbar_arrive(smem_u32(&ctl->cempty[cs]));
+                    mbar_arrive_cluster_light(smem_u32(&ctl->full[ring.s]), 0);
+                    mbar_arrive(smem_u32(&ctl->cempty[ring.cs]));
                 }
+                ring.advance();
             }
             if (__any_sync(0xffffffffu, ctl->abort_flag != 0)) ok = false;
         }
@@ -389,6 +441,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         const int et = threadIdx.x - EPI_WARP0 * 32;               // 0..127, for the cooperative column staging
         const int row = ew * 32 + lane;                            // accumulator row within the CTA
         const float zoff = (A_BITS == 8) ? 128.f : 8.f;            // the A operand is fed as q - 128 / q - 8
+        const bool has_ws = p.wscale != nullptr, has_bias = p.bias != nullptr;
         uint32_t t = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
             const int m0 = (tile % tiles_m) * 2 * BM_CTA + (int)rank * BM_CTA, n0 = (tile / tiles_m) * BN;
@@ -397,10 +450,10 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             float (*col)[BN] = ctl->col[buf];
             for (int c = et; c < BN; c += NUM_EPI_WARPS * 32) {
                 const int n = n0 + c;
-                const bool ok = n < p.N;
-                col[0][c] = ok ? __ldg(p.wsum + n) : 0.f;
-                col[1][c] = (ok && p.wscale) ? __ldg(p.wscale + n) : 1.f;
-                col[2][c] = (ok && p.bias) ? __ldg(p.bias + n) : 0.f;
+                const bool okc = n < p.N;
+                col[0][c] = okc ? __ldg(p.wsum + n) : 0.f;
+                if (has_ws) col[1][c] = okc ? __ldg(p.wscale + n) : 1.f;
+                if (has_bias) col[2][c] = okc ? __ldg(p.bias + n) : 0.f;
             }
             // barrier over the four epilogue warps; they leave together once any of them has seen the abort flag
             if (bar_or_epilogue(ctl->abort_flag != 0)) break;
@@ -408,7 +461,8 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             const bool row_ok = m < p.M;
             const float sm = row_ok ? __ldg(p.a_scale + m) : 0.f;
             const float zm = row_ok ? (float)__ldg(p.a_zp + m) + zoff : 0.f;
-            const bool okw = mbar_wait_warp(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, &ctl->abort_flag, p.status, 8);
+            const f32x2 SM = pack2(sm, sm), ZM = pack2(zm, zm);
+            const bool okw = mbar_wait_warp<500>(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, &ctl->abort_flag, p.status, 8);
             tc_fence_after();
             if (okw) {
 #pragma unroll 1
@@ -418,30 +472,49 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                     tc_ld32(tmem_base + ((uint32_t)(ew * 32) << 16) + (uint32_t)(buf * BN + c0), acc);
                     tc_wait_ld();
                     if (row_ok) {
-                        float y[32];
+                        // y = s_m * (acc + z_m * wsum_n) [* wscale_n] [+ bias_n], two columns per instruction
+                        f32x2 y[16];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            y[j] = fmaf(sm * fmaf(zm, col[0][c0 + j], __uint_as_float(acc[j])), col[1][c0 + j], col[2][c0 + j]);
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 ws = *reinterpret_cast<const float4*>(&col[0][c0 + 4 * j]);
+                            f32x2 a0 = fma2(ZM, pack2(ws.x, ws.y), pack2(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1])));
+                            f32x2 a1 = fma2(ZM, pack2(ws.z, ws.w), pack2(__uint_as_float(acc[4 * j + 2]), __uint_as_float(acc[4 * j + 3])));
+                            a0 = mul2(a0, SM); a1 = mul2(a1, SM);
+                            if (has_ws) {
+                                const float4 sc = *reinterpret_cast<const float4*>(&col[1][c0 + 4 * j]);
+                                a0 = mul2(a0, pack2(sc.x, sc.y)); a1 = mul2(a1, pack2(sc.z, sc.w));
+                            }
+                            if (has_bias) {
+                                const float4 bi = *reinterpret_cast<const float4*>(&col[2][c0 + 4 * j]);
+                                a0 = add2(a0, pack2(bi.x, bi.y)); a1 = add2(a1, pack2(bi.z, bi.w));
+                            }
+                            y[2 * j] = a0; y[2 * j + 1] = a1;
+                        }
                         const int nvalid = min(32, p.N - (n0 + c0));
                         if (p.y_dtype == LRQ_F32) {
                             float* dst = static_cast<float*>(p.Y) + (size_t)m * p.ldy + n0 + c0;
                             if (nvalid == 32) {
 #pragma unroll
                                 for (int j = 0; j < 8; ++j)
-                                    reinterpret_cast<float4*>(dst)[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+                                    reinterpret_cast<ulonglong2*>(dst)[j] = make_ulonglong2(y[2 * j], y[2 * j + 1]);
                             } else {
 #pragma unroll
-                                for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = y[j];
+                                for (int j = 0; j < 16; ++j) {
+                                    float a, b; unpack2(y[j], a, b);
+                                    if (2 * j < nvalid) dst[2 * j] = a;
+                                    if (2 * j + 1 < nvalid) dst[2 * j + 1] = b;
+                                }
                             }
                         } else {
                             uint32_t h[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
+                                float a, b; unpack2(y[j], a, b);
                                 if (p.y_dtype == LRQ_BF16) {
-                                    __nv_bfloat162 v = __floats2bfloat162_rn(y[2 * j], y[2 * j + 1]);
+                                    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
                                     h[j] = *reinterpret_cast<uint32_t*>(&v);
                                 } else {
-                                    __half2 v = __floats2half2_rn(y[2 * j], y[2 * j + 1]);
+                                    __half2 v = __floats2half2_rn(a, b);
                                     h[j] = *reinterpret_cast<uint32_t*>(&v);
                                 }
                             }

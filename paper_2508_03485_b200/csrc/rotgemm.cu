@@ -74,7 +74,7 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
-                    ok = mbar_wait(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, status, 11);
+                    ok = mbar_wait<100>(smem_u32(&ctl->empty[s]), ((it / STAGES) & 1) ^ 1, &ctl->abort_flag, status, 11);
                     if (!ok) break;
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     mbar_arrive_expect_tx(bar, STAGE_TX_BYTES);
@@ -102,13 +102,13 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++t) {
                 const int buf = t & 1;
-                ok = mbar_wait(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, status, 12);
+                ok = mbar_wait<64>(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, status, 12);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
-                    ok = mbar_wait(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, status, 13);
+                    ok = mbar_wait<32>(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, status, 13);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(sA + s * A_STAGE_BYTES), b_addr = smem_u32(sB + s * B_STAGE_BYTES);
@@ -132,7 +132,7 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
             const int buf = t & 1;
             const int m = m0 + row;
-            const bool okw = mbar_wait(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, &ctl->abort_flag, status, 14);
+            const bool okw = mbar_wait<500>(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, &ctl->abort_flag, status, 14);
             tc_fence_after();
             if (okw) {
 #pragma unroll 1

@@ -65,11 +65,15 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 }
 
 // Bounded wait.  Returns false (after raising *abort_flag and recording `code` in *status) when the
-// phase never completed, or as soon as another thread of the CTA has raised the flag.
+// phase never completed, or as soon as another thread of the CTA has raised the flag.  Between polls the
+// thread sleeps SLEEP_NS nanoseconds: a warp that spins on try_wait competes for issue slots with the
+// warps that do the work, and most waiters here (epilogue, TMA producer) are far from the critical path.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     do {
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     } while (clock64() - t0 < kWaitCycles);
@@ -80,14 +84,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // The same for a whole (converged) warp.  Every lane waits on the barrier itself (a lane that has not
 // observed the phase has no ordering against the asynchronous writes it guards), then the lanes agree
 // on one answer, so that warp-level synchronisation after the wait stays convergent when a wait expires.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
-    const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
+    const bool ok = mbar_wait<SLEEP_NS>(bar, parity, abort_flag, status, code);
     return __all_sync(0xffffffffu, ok);
 }
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     const long long t0 = clock64();
     do {
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
         if (mbar_try_wait_cluster(bar, parity)) return true;
         if (*abort_flag) return false;
     } while (clock64() - t0 < kWaitCycles);
