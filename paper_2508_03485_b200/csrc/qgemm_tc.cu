@@ -89,23 +89,45 @@ __device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4)); }
 
 // ---- activation codes -> bf16 ---------------------------------------------------------------------
+// Constants of the expansions, held in registers: an instruction encodes at most one immediate, so a
+// three-input logic operation or a byte permute with two constant operands would otherwise be split in two.
+struct ExpandConst {
+    uint32_t k7f, k43, k80, kc3, k4343;
+    __device__ ExpandConst() {
+        asm volatile("mov.u32 %0, 0x007F007F;" : "=r"(k7f));
+        asm volatile("mov.u32 %0, 0x43004300;" : "=r"(k43));
+        asm volatile("mov.u32 %0, 0x00800080;" : "=r"(k80));
+        asm volatile("mov.u32 %0, 0xC380C380;" : "=r"(kc3));
+        asm volatile("mov.u32 %0, 0x43434343;" : "=r"(k4343));
+    }
+};
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {     // (a & b) | c
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t b, uint32_t c) {    // (a & b) ^ c
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
 // 8-bit: four codes per word -> bf16 of (q - 128).  0x4300|x7 is 128 + x7; adding -256 (bit 7 clear)
 // or -128 (bit 7 set) gives q - 128 exactly.
-__device__ __forceinline__ void expand_a8(uint32_t w, uint32_t& o01, uint32_t& o23) {
+__device__ __forceinline__ void expand_a8(uint32_t w, const ExpandConst& k, uint32_t& o01, uint32_t& o23) {
     const uint32_t p01 = prmt(w, 0u, 0x4140u), p23 = prmt(w, 0u, 0x4342u);
-    o01 = add_bf16x2((p01 & 0x007F007Fu) | 0x43004300u, (p01 & 0x00800080u) ^ 0xC380C380u);
-    o23 = add_bf16x2((p23 & 0x007F007Fu) | 0x43004300u, (p23 & 0x00800080u) ^ 0xC380C380u);
+    o01 = add_bf16x2(and_or(p01, k.k7f, k.k43), and_xor(p01, k.k80, k.kc3));
+    o23 = add_bf16x2(and_or(p23, k.k7f, k.k43), and_xor(p23, k.k80, k.kc3));
 }
 // 4-bit: eight codes per word -> bf16 of (q - 8): 0x4300 | q is 128 + q, and 128 + q - 136 is exact.
 // The eight elements come out in the order k = 0,2, 4,6, 1,3, 5,7 within the word (one byte permute per
 // pair instead of a permute and an OR); the weight decode of 4-bit-activation layers emits the same order,
 // and a contraction does not care in which order k is summed as long as both operands agree.
-__device__ __forceinline__ void expand_a4(uint32_t w, uint32_t* o) {
+__device__ __forceinline__ void expand_a4(uint32_t w, const ExpandConst& k, uint32_t* o) {
     const uint32_t lo = w & 0x0F0F0F0Fu, hi = (w >> 4) & 0x0F0F0F0Fu;      // even / odd codes, one per byte
-    o[0] = add_bf16x2(prmt(lo, 0x43434343u, 0x4140u), 0xC308C308u);        // codes 0, 2
-    o[1] = add_bf16x2(prmt(lo, 0x43434343u, 0x4342u), 0xC308C308u);        // codes 4, 6
-    o[2] = add_bf16x2(prmt(hi, 0x43434343u, 0x4140u), 0xC308C308u);        // codes 1, 3
-    o[3] = add_bf16x2(prmt(hi, 0x43434343u, 0x4342u), 0xC308C308u);        // codes 5, 7
+    o[0] = add_bf16x2(prmt(lo, k.k4343, 0x4140u), 0xC308C308u);            // codes 0, 2
+    o[1] = add_bf16x2(prmt(lo, k.k4343, 0x4342u), 0xC308C308u);            // codes 4, 6
+    o[2] = add_bf16x2(prmt(hi, k.k4343, 0x4140u), 0xC308C308u);            // codes 1, 3
+    o[3] = add_bf16x2(prmt(hi, k.k4343, 0x4342u), 0xC308C308u);            // codes 5, 7
 }
 
 // ---- TLQ codes -> bf16 through the row's level table ------------------------------------------------
@@ -395,6 +417,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
 #pragma unroll
         for (int j = 0; j < OUT_CH; ++j) off[j] = swz(row0, OUT_CH * cc + j);
         const uint32_t sA0 = smem_u32(sA), sAc0 = smem_u32(sAc) + (uint32_t)tl * 16;
+        const ExpandConst kx;
         RingPos ring(grp);
         uint32_t it0 = 0;
         bool ok = true;
@@ -416,10 +439,10 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                     const uint4 cw = cws[i];
                     uint32_t o[4 * OUT_CH];
                     if constexpr (A_BITS == 8) {
-                        expand_a8(cw.x, o[0], o[1]); expand_a8(cw.y, o[2], o[3]);
-                        expand_a8(cw.z, o[4], o[5]); expand_a8(cw.w, o[6], o[7]);
+                        expand_a8(cw.x, kx, o[0], o[1]); expand_a8(cw.y, kx, o[2], o[3]);
+                        expand_a8(cw.z, kx, o[4], o[5]); expand_a8(cw.w, kx, o[6], o[7]);
                     } else {
-                        expand_a4(cw.x, o); expand_a4(cw.y, o + 4); expand_a4(cw.z, o + 8); expand_a4(cw.w, o + 12);
+                        expand_a4(cw.x, kx, o); expand_a4(cw.y, kx, o + 4); expand_a4(cw.z, kx, o + 8); expand_a4(cw.w, kx, o + 12);
                     }
 #pragma unroll
                     for (int j = 0; j < OUT_CH; ++j)      // ROWS_PER_TASK rows further down: whole 1024-byte groups
