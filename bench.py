@@ -210,8 +210,29 @@ def run_cuda(args):
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
+    def step_direct():
+        P.lrq_qlinear_stack(plan, ws, torch.cuda.current_stream())
+
+    # The step is captured once into a CUDA graph and replayed: the path is a fixed sequence of launches, and a
+    # replay removes the host-side launch gaps between them (--no-graph times the plain stream-ordered calls).
+    graph = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            for _ in range(2):
+                step_direct()            # first-call set-up (function attributes, occupancy queries) happens outside the capture
+        stream.wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step_direct()
+
     def step():
-        P.lrq_qlinear_stack(plan, ws, stream)
+        if graph is not None:
+            graph.replay()
+        else:
+            step_direct()
 
     def timed(fn, n, flush_between=True):
         evs = []
@@ -311,6 +332,7 @@ def run_cuda(args):
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(args.config), "layers": len(specs), "out_dtype": "f32",
                        "l2": "flushed between timed steps (512 MiB fill outside the timed events)",
+                       "launch": "one CUDA graph replay per step" if graph is not None else "stream-ordered launches",
                        "parallelism": f"replicated batch x{world}, no collective"},
             "tokens_per_s": world * tokens / (ms_step * 1e-3),
             "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -364,6 +386,16 @@ def run_kernel(args):
     for _ in range(max(1, args.warmup)):
         fn()
     torch.cuda.synchronize()
+    if not args.no_graph and args.kernel != "tlq":
+        call = fn
+        if args.kernel == "rotq":
+            call = lambda: P.lrq_rotate_quantize_act(X, kind, s.a_bits, s.had_block, R, workspace=ws, out=rq)
+        elif args.kernel == "qgemm":
+            call = lambda: P.lrq_qgemm_codes(L, rq[0], rq[1], rq[2], P.F32, args.gemm_impl, Y)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            call()
+        fn = g.replay
     ts = []
     for _ in range(args.steps):
         flush.fill_(1)
@@ -388,6 +420,7 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--gemm-impl", type=int, default=0, choices=[0, 1],
                     help="kernel timed alone for the roofline object: 0 tcgen05, 1 CUDA-core baseline")
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph replay of the step")
     ap.add_argument("--kernel", default=None, choices=["rotq", "qgemm", "tlq"], help="time one kernel only")
     ap.add_argument("--layer", type=int, default=0, help="layer index of the workload for --kernel")
     ap.add_argument("--tokens", type=int, default=0, help="override M for --kernel")

@@ -55,8 +55,13 @@ extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long 
         const size_t need = lrq_act_workspace_bytes(M, K, p);
         if (!workspace || workspace_bytes < need || !lrq_aligned(workspace, 256)) return LRQ_ERR_WORKSPACE;
         float* Yr = static_cast<float*>(workspace);
-        st = lrq_launch_rotgemm(X, M, K, ldx, p->R_bf16, Yr, stream);
+        // the rotation leaves each token's extremes in the scale / zero-point outputs (as integers); the
+        // quantizer reads them and then writes the real values there
+        bool have_ext = false;
+        st = lrq_launch_rotgemm(X, M, K, ldx, p->R_bf16, Yr, reinterpret_cast<int*>(a_scale), reinterpret_cast<int*>(a_zp),
+                                &have_ext, stream);
         if (st != LRQ_OK) return st;
+        if (have_ext) return lrq_launch_quantize_f32_ext(Yr, M, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
         return lrq_launch_quantize_f32(Yr, M, K, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
     }
     const int B = p->kind == LRQ_ROT_HADAMARD ? p->had_block : 1;

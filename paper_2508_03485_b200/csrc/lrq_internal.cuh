@@ -34,8 +34,20 @@ lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B
                                     uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
 lrq_status lrq_launch_quantize_f32(const float* Y, int M, int K, long ldy, int a_bits, int mode,
                                    uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
-// rotgemm.cu : Y[M,K] (fp32) = X[M,K] (bf16) . R[K,K] (bf16)
-lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y, cudaStream_t st);
+// rotgemm.cu : Y[M,K] (fp32) = X[M,K] (bf16) . R[K,K] (bf16).  When the tensor-core kernel runs it also leaves
+// every row's minimum and maximum in ext_min[M] / ext_max[M] as order-preserving integers (*have_ext = true).
+lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y,
+                              int* ext_min, int* ext_max, bool* have_ext, cudaStream_t st);
+// rotq.cu : per-token quantization of fp32 rows whose extremes are already known (ext_min / ext_max alias the
+// scale / zero-point outputs: each row's extremes are read before its results are written).
+lrq_status lrq_launch_quantize_f32_ext(const float* Y, int M, int K, int a_bits, int mode, uint8_t* codes,
+                                       float* scale, int32_t* zp, cudaStream_t st);
+
+#ifdef __CUDACC__
+// Order-preserving map between fp32 and int32 (and back), so that integer min/max reductions serve floats.
+__device__ __forceinline__ int lrq_ordered_int(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
+__device__ __forceinline__ float lrq_ordered_float(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+#endif
 // qgemm_simple.cu / qgemm_tc.cu
 lrq_status lrq_launch_qgemm_simple(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                                    const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);

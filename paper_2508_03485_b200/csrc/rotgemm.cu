@@ -1,6 +1,8 @@
 // Outlier-aware rotation y = x . R (Sec. 4.2, Eq. 12, second case) as a dense contraction on the
 // 5th-generation tensor cores: X bf16 [M,K] times R bf16 [K,K] into an fp32 scratch that the
 // per-token quantizer then reads.  bf16 x bf16 products are exact in fp32; sums are accumulated in fp32.
+// The epilogue also folds every row's minimum and maximum into two integer arrays (atomic min / max on
+// order-preserving images), so that the quantizer that follows is a single streaming pass.
 //
 // Persistent CTA per SM over 128 x 256 output tiles, 64-deep k-blocks, a 4-stage TMA pipeline:
 //   warp 0      one lane issues the TMA tile loads (X: K-major box 64 x 128; R: four 64 x 64 boxes, each
@@ -40,7 +42,7 @@ constexpr uint32_t IDESC = umma_idesc_bf16(BM, BN, /*a_mn_major=*/false, /*b_mn_
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
-                  float* __restrict__ Y, int M, int K, int* status) {
+                  float* __restrict__ Y, int M, int K, int* __restrict__ ext_min, int* __restrict__ ext_max, int* status) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     unsigned char* sA = base;
@@ -134,6 +136,7 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             const int m = m0 + row;
             const bool okw = mbar_wait<500>(smem_u32(&ctl->tmem_full[buf]), (t >> 1) & 1, &ctl->abort_flag, status, 14);
             tc_fence_after();
+            float mn = INFINITY, mx = -INFINITY;         // extremes of this row over the tile's columns
             if (okw) {
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -147,9 +150,18 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
                                 reinterpret_cast<uint4*>(dst)[j] = make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+#pragma unroll
+                            for (int j = 0; j < 32; j += 2) {
+                                asm("min.f32 %0, %0, %1, %2;" : "+f"(mn) : "f"(__uint_as_float(acc[j])), "f"(__uint_as_float(acc[j + 1])));
+                                asm("max.f32 %0, %0, %1, %2;" : "+f"(mx) : "f"(__uint_as_float(acc[j])), "f"(__uint_as_float(acc[j + 1])));
+                            }
                         } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (n0 + c0 + j < K) dst[j] = __uint_as_float(acc[j]);
+                            for (int j = 0; j < 32; ++j)
+                                if (n0 + c0 + j < K) {
+                                    const float v = __uint_as_float(acc[j]);
+                                    dst[j] = v; mn = fminf(mn, v); mx = fmaxf(mx, v);
+                                }
                         }
                     }
                 }
@@ -157,6 +169,10 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[buf]));
+            if (okw && m < M && ext_min) {                // fold this tile's share into the row's extremes
+                atomicMin(ext_min + m, lrq_ordered_int(mn));
+                atomicMax(ext_max + m, lrq_ordered_int(mx));
+            }
             if (ctl->abort_flag) break;
         }
     }
@@ -216,7 +232,9 @@ rotgemm_simple_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ld
 
 }  // namespace
 
-lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y, cudaStream_t st) {
+lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y,
+                              int* ext_min, int* ext_max, bool* have_ext, cudaStream_t st) {
+    if (have_ext) *have_ext = false;
     // TMA needs 16-byte aligned bases and row pitches; the fp32 rows are stored with 128-bit stores
     const bool tc_ok = (K % 8) == 0 && (ldx % 8) == 0 && lrq_aligned(X, 16) && lrq_aligned(R, 16) && lrq_aligned(Y, 16);
     if (tc_ok) {
@@ -232,7 +250,14 @@ lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void*
         LRQ_CUDA_TRY(cudaGetDevice(&dev));
         LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         const int tiles = ((M + BM - 1) / BM) * ((K + BN - 1) / BN);
-        rotgemm_tc_kernel<<<tiles < sms ? tiles : sms, NUM_THREADS, SMEM_BYTES, st>>>(tmX, tmR, Y, M, K, lrq_status_word());
+        const bool ext = ext_min && ext_max;
+        if (ext) {          // identity elements of the integer min / max: bytes 0x7f.. (a huge float), 0x80.. (a hugely negative one)
+            LRQ_CUDA_TRY(cudaMemsetAsync(ext_min, 0x7f, (size_t)M * sizeof(int), st));
+            LRQ_CUDA_TRY(cudaMemsetAsync(ext_max, 0x80, (size_t)M * sizeof(int), st));
+        }
+        rotgemm_tc_kernel<<<tiles < sms ? tiles : sms, NUM_THREADS, SMEM_BYTES, st>>>(tmX, tmR, Y, M, K, ext ? ext_min : nullptr,
+                                                                                    ext ? ext_max : nullptr, lrq_status_word());
+        if (have_ext) *have_ext = ext;
         LRQ_CUDA_TRY(cudaGetLastError());
         return LRQ_OK;
     }

@@ -173,10 +173,6 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm(
 __device__ __forceinline__ float min3(float a, float b, float c) { float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
 __device__ __forceinline__ float max3(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
 
-// Order-preserving map between fp32 and int32 (and back), so that integer min/max reductions serve floats.
-__device__ __forceinline__ int ordered_int(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
-__device__ __forceinline__ float ordered_float(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
-
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
     uint4 r;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -351,7 +347,7 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
         for (int i = 1; i < NP; ++i) { float x, y; unpack2(P[i], x, y); mn = min3(mn, x, y); mx = max3(mx, x, y); }
         int* slot = ext + (it % 3) * 2 * tok_per_cta + 2 * tl;
         {
-            const int imn = __reduce_min_sync(seg_mask, ordered_int(mn)), imx = __reduce_max_sync(seg_mask, ordered_int(mx));
+            const int imn = __reduce_min_sync(seg_mask, lrq_ordered_int(mn)), imx = __reduce_max_sync(seg_mask, lrq_ordered_int(mx));
             if (seg_leader) { atomicMin(slot, imn); atomicMax(slot + 1, imx); }
         }
         __syncthreads();
@@ -361,7 +357,7 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
             float sc = 0.f; int z = 0;
             t.inv = 0.f; t.negz = 0.f;
             if (seg_leader) {
-                const float a = ordered_float(slot[0]), b = ordered_float(slot[1]);
+                const float a = lrq_ordered_float(slot[0]), b = lrq_ordered_float(slot[1]);
                 t = token_params_fast(a, b, A_BITS, mode, 1.0 / sqrt((double)(1 << LOG2B)), &sc, &z);
                 if (j == 0 && live) { scale[m] = sc; zp[m] = z; }
             }
@@ -404,7 +400,67 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Quantizer of already rotated fp32 rows whose extremes are known (dense path: the rotation GEMM's epilogue
+// found them).  One warp per token, grid-stride; lane 0 works out the step and zero-point, then the warp
+// streams the row: 32 bytes in (one 256-bit load), 8 or 4 code bytes out per lane and step.
+// ext_min / ext_max alias scale / zp: the warp reads its row's extremes before it writes the results.
+// ------------------------------------------------------------------------------------------------
+template <int A_BITS>
+__global__ void __launch_bounds__(256)
+quant_rows_f32_kernel(const float* __restrict__ Y, int M, int K, int mode, uint8_t* __restrict__ codes,
+                      float* scale, int32_t* zp) {
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; m < M; m += warps) {
+        TokenQ t;
+        t.inv = 0.f; t.negz = 0.f;
+        if (lane == 0) {
+            const float mn = lrq_ordered_float(reinterpret_cast<const int*>(scale)[m]);
+            const float mx = lrq_ordered_float(reinterpret_cast<const int*>(zp)[m]);
+            float sc; int32_t z;
+            t = token_params_fast(mn, mx, A_BITS, mode, 1.0, &sc, &z);
+            scale[m] = sc; zp[m] = z;
+        }
+        t.inv = __shfl_sync(0xffffffffu, t.inv, 0);
+        t.negz = __shfl_sync(0xffffffffu, t.negz, 0);
+        const f32x2 INV = pack2(t.inv, t.inv), NEGZ = pack2(t.negz, t.negz);
+        const float* row = Y + (size_t)m * K;
+        for (int c = lane; c < (K >> 3); c += 32) {
+            uint32_t r[8];
+            asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                         : "l"(row + 8 * c));
+            int q[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float x, y;
+                unpack2(fma2(pack2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), INV, NEGZ), x, y);
+                q[2 * i] = __float2int_rn(x); q[2 * i + 1] = __float2int_rn(y);
+            }
+            if (A_BITS == 8)
+                *reinterpret_cast<uint2*>(codes + (size_t)m * K + 8 * c) = make_uint2(pack_u8x4(q[0], q[1], q[2], q[3]), pack_u8x4(q[4], q[5], q[6], q[7]));
+            else
+                *reinterpret_cast<uint32_t*>(codes + (((size_t)m * K) >> 1) + 4 * c) = pack_u4x8(q);
+        }
+    }
+}
+
 }  // namespace
+
+lrq_status lrq_launch_quantize_f32_ext(const float* Y, int M, int K, int a_bits, int mode, uint8_t* codes,
+                                       float* scale, int32_t* zp, cudaStream_t st) {
+    if (!lrq_aligned(Y, 32)) return LRQ_ERR_INVALID_ARG;          // rows are K*4 bytes with K % 8 == 0: 32-byte aligned chunks
+    int dev = 0, sms = 0;
+    LRQ_CUDA_TRY(cudaGetDevice(&dev));
+    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int blocks_needed = (M + 7) / 8;                        // 8 warps per CTA, one token per warp and step
+    const int grid = blocks_needed < sms * 8 ? blocks_needed : sms * 8;
+    if (a_bits == 8) quant_rows_f32_kernel<8><<<grid, 256, 0, st>>>(Y, M, K, mode, codes, scale, zp);
+    else quant_rows_f32_kernel<4><<<grid, 256, 0, st>>>(Y, M, K, mode, codes, scale, zp);
+    LRQ_CUDA_TRY(cudaGetLastError());
+    return LRQ_OK;
+}
 
 static lrq_status launch_generic(bool f32, const void* X, int M, int K, long ldx, int log2B, int a_bits, int mode,
                                  uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st) {
