@@ -151,6 +151,16 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------------------------------ ranks
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (the per-step time of a multi-GPU run is the
+    slowest rank's).  `dist` is torch.distributed with an initialised process group; works with gloo on CPU."""
+    import torch
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
 # ------------------------------------------------------------------------------------------ CUDA arm
 def run_cuda(args):
     import torch
@@ -284,9 +294,7 @@ def run_cuda(args):
     clocks = sampler.stop() if rank == 0 else None
 
     if world > 1:
-        t = torch.tensor([ms_step, e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, e2e_ms = float(t[0]), float(t[1])
+        ms_step, e2e_ms = max_over_ranks([ms_step, e2e_ms], dist, dev)
 
     flops = layer_flops(specs)
     tokens = sum(s.M for s in specs) / len(specs) if args.config != 4 else specs[0].M

@@ -184,3 +184,62 @@ def test_qlinear_stack_matches_single_calls(P):
     torch.cuda.synchronize()
     for y, r in zip(Ys, refs):
         assert torch.equal(y, r)
+
+
+# ------------------------------------------------------------------ tensor-core kernel at full size
+@pytest.mark.parametrize("cfg,li", [(1, 0), (2, 0), (3, 1)])
+def test_qgemm_tensor_core_matches_cuda_core_everywhere(P, cfg, li):
+    # Every output element of the tcgen05 kernel against the plain CUDA-core kernel of the same library on a
+    # BASELINE-sized layer: several tiles per CTA pair, grouped and per-channel tables, 4- and 8-bit codes.
+    # The oracle checks sampled rows elsewhere; this one looks at all of them, twice (a hand-over race
+    # between the kernel's warps shows up as a few wrong tiles that differ from run to run).
+    spec = config_layers(cfg)[li]
+    layer, tl = PU.gpu_layer(spec, spec.weights(), P)
+    X = PU.bf16_to_device(spec.activations())
+    kind = P.ROT_HADAMARD
+    q, s, z = P.lrq_rotate_quantize_act(X, kind, spec.a_bits, spec.had_block)
+    ref = P.lrq_qgemm_codes(layer, q, s, z, P.F32, 1)
+    first = None
+    for _ in range(3):
+        Y = P.lrq_qgemm_codes(layer, q, s, z, P.F32, 0)
+        torch.cuda.synchronize()
+        assert P.lrq_device_status() == 0
+        rms = ref.pow(2).mean().sqrt()
+        assert ((Y - ref).abs().max() / rms).item() <= 2e-3          # fp32 summation order only
+        if first is None:
+            first = Y.clone()
+        else:
+            assert torch.equal(Y, first)                             # fixed accumulation order: bit-identical
+    layer.close()
+
+
+def test_qlinear_stack_replays_from_a_cuda_graph(P):
+    # The stack is a fixed sequence of launches (kernels with by-value tensor maps, two memsets for a dense
+    # rotation): captured once, replayed on new activations, it must give what direct calls give.
+    specs = [LayerSpec("a", 61, 200, 1152, 264, 4, 8, 0, "hadamard", 128),
+             LayerSpec("b", 62, 130, 512, 136, 3, 4, 128, "dense", 0)]
+    layers, Xs, Ys = [], [], []
+    for sp in specs:
+        layer, _ = PU.gpu_layer(sp, sp.weights(), P)
+        layers.append(layer)
+        Xs.append(PU.bf16_to_device(sp.activations()))
+        Ys.append(torch.zeros((sp.M, sp.N), dtype=torch.float32, device="cuda"))
+    plan = P.StackPlan(layers, Xs, Ys, P.F32)
+    ws = torch.empty(plan.need, dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        P.lrq_qlinear_stack(plan, ws)                # first-call set-up happens outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        P.lrq_qlinear_stack(plan, ws)
+    for seed in (71, 72):
+        for sp, X in zip(specs, Xs):
+            X.copy_(PU.bf16_to_device(make_activations(seed, sp.M, sp.K, n_salient=8 if sp.rot == "dense" else 0)))
+        g.replay()
+        torch.cuda.synchronize()
+        for layer, X, Y in zip(layers, Xs, Ys):
+            assert torch.equal(Y, P.lrq_qlinear(layer, X, P.F32))
+    assert P.lrq_device_status() == 0
