@@ -33,6 +33,18 @@ sys.path.insert(0, ROOT)
 
 from lrq_workloads import bf16_bits_to_f64, config_layers, default_clip_grid  # noqa: E402
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/, keyed by the kernel and layer the roofline object describes.  A key is dropped (traffic: null) when its
+# kernel changes after the capture.
+NCU_TRAFFIC_BYTES = {
+    "qgemm cfg1 fc1": 7.83e6 + 23.37e6,
+    "qgemm cfg3 fc1": 27.03e6 + 174.04e6,
+    "qgemm cfg4 b0.fc1": 123.76e6 + 552.45e6,
+    "rotq cfg1 fc2": None,                      # 57 MB case not captured; the M = 32768 capture of the same layer shape:
+    "rotq cfg4 b0.fc2": 302.28e6 + 123.51e6,
+    "rotq cfg3 fc2": 113.83e6 + 16.29e6,
+}
+
 METRIC = "qlinear_tflops"
 UNIT = "TFLOP/s"
 ORACLE_SAMPLE_TOKENS = 128
@@ -320,11 +332,14 @@ def run_cuda(args):
         rot_gbs = rot_bytes / (rot_ms * 1e-3) / 1e9
         roofline = {"kernel": f"qgemm {s.name} {s.M}x{s.N}x{s.K} W{s.w_bits}A{s.a_bits}", "bound": "tensor",
                     "achieved": gemm_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": gemm_tf / peaks["bf16_tflops"], "traffic": None, "peak_source": peaks["source"] + " burst bf16",
+                    "frac": gemm_tf / peaks["bf16_tflops"], "traffic": NCU_TRAFFIC_BYTES.get(f"qgemm cfg{args.config} {s.name}"),
+                    "traffic_unit": "bytes per launch (ncu dram read + write)", "algorithmic_flops": 2.0 * s.M * s.N * s.K,
+                    "peak_source": peaks["source"] + " burst bf16",
                     "ms": gemm_ms}
         roofline_rotq = {"kernel": f"rotq {sr.name} {sr.M}x{sr.K} B{sr.had_block} A{sr.a_bits}", "bound": "hbm",
                          "achieved": rot_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rot_gbs / peaks["hbm_gbs"],
-                         "traffic": None, "peak_source": peaks["source"], "ms": rot_ms, "algorithmic_bytes": rot_bytes}
+                         "traffic": NCU_TRAFFIC_BYTES.get(f"rotq cfg{args.config} {sr.name}"), "peak_source": peaks["source"],
+                         "ms": rot_ms, "algorithmic_bytes": rot_bytes}
         # ---- CPU baseline: the oracle, as it stands, on a bounded token sample
         import oracle as orc
         orc.build()
