@@ -68,8 +68,10 @@ struct __align__(16) SharedCtl {
     alignas(16) float col[2][3][BN];   // per TMEM buffer: wsum, wscale, bias of the tile's columns (read as float4)
 };
 
+constexpr int EPI_TILE_BYTES = 32 * 32 * 4;         // one epilogue warp's 32 x 32 fp32 chunk, for the row/column trade
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
-                              (size_t)CSTAGES * (AC_STAGE_BYTES + WC_STAGE_BYTES) + sizeof(SharedCtl);
+                              (size_t)CSTAGES * (AC_STAGE_BYTES + WC_STAGE_BYTES) + sizeof(SharedCtl) +
+                              (size_t)NUM_EPI_WARPS * EPI_TILE_BYTES;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 constexpr uint32_t IDESC = umma_idesc_bf16(2 * BM_CTA, BN, false, false);
@@ -230,6 +232,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
     unsigned char* sAc = sB + STAGES * B_STAGE_BYTES;               // CSTAGES x 8 KB
     unsigned char* sWc = sAc + CSTAGES * AC_STAGE_BYTES;            // CSTAGES x 4 KB
     SharedCtl* ctl = reinterpret_cast<SharedCtl*>(sWc + CSTAGES * WC_STAGE_BYTES);
+    unsigned char* sEpi = reinterpret_cast<unsigned char*>(ctl) + sizeof(SharedCtl);   // NUM_EPI_WARPS x 4 KB
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                       // 0: issues the MMAs, 1: its peer
@@ -494,9 +497,10 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                     uint32_t acc[32];
                     tc_ld32(tmem_base + ((uint32_t)(ew * 32) << 16) + (uint32_t)(buf * BN + c0), acc);
                     tc_wait_ld();
+                    f32x2 yq[16];
                     if (row_ok) {
                         // y = s_m * (acc + z_m * wsum_n) [* wscale_n] [+ bias_n], two columns per instruction
-                        f32x2 y[16];
+                        f32x2* y = yq;
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             const float4 ws = *reinterpret_cast<const float4*>(&col[0][c0 + 4 * j]);
@@ -514,20 +518,16 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                             y[2 * j] = a0; y[2 * j + 1] = a1;
                         }
                         const int nvalid = min(32, p.N - (n0 + c0));
-                        if (p.y_dtype == LRQ_F32) {
+                        if (p.y_dtype == LRQ_F32 && nvalid < 32) {
                             float* dst = static_cast<float*>(p.Y) + (size_t)m * p.ldy + n0 + c0;
-                            if (nvalid == 32) {
 #pragma unroll
-                                for (int j = 0; j < 8; ++j)
-                                    reinterpret_cast<ulonglong2*>(dst)[j] = make_ulonglong2(y[2 * j], y[2 * j + 1]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) {
-                                    float a, b; unpack2(y[j], a, b);
-                                    if (2 * j < nvalid) dst[2 * j] = a;
-                                    if (2 * j + 1 < nvalid) dst[2 * j + 1] = b;
-                                }
+                            for (int j = 0; j < 16; ++j) {
+                                float a, b; unpack2(y[j], a, b);
+                                if (2 * j < nvalid) dst[2 * j] = a;
+                                if (2 * j + 1 < nvalid) dst[2 * j + 1] = b;
                             }
+                        } else if (p.y_dtype == LRQ_F32) {
+                            // handled below by the whole warp (rows past M take part in the exchange, not in the stores)
                         } else {
                             uint32_t h[16];
 #pragma unroll
@@ -549,6 +549,34 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                             } else {
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = (uint16_t)(h[j >> 1] >> (16 * (j & 1)));
+                            }
+                        }
+                    }
+                    if (p.y_dtype == LRQ_F32 && n0 + c0 + 32 <= p.N) {
+                        // A lane holds 32 consecutive outputs of its own row; stored as they are, every store would
+                        // touch 32 different rows, half a sector each.  The warp trades rows for columns through a
+                        // 4 KB tile (16-byte chunk index XOR-ed with the row's low bits: conflict-free both ways), so
+                        // that each store writes four rows' whole 128-byte lines.
+                        const uint32_t tile = smem_u32(sEpi) + (uint32_t)ew * EPI_TILE_BYTES;
+                        __syncwarp();
+                        if (row_ok) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float a, b, c2, d;
+                                unpack2(yq[2 * j], a, b); unpack2(yq[2 * j + 1], c2, d);
+                                sts128(tile + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4)), __float_as_uint(a), __float_as_uint(b),
+                                       __float_as_uint(c2), __float_as_uint(d));
+                            }
+                        }
+                        __syncwarp();
+                        const int rsub = lane >> 3, jq = lane & 7;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int r = 4 * i + rsub, mr = m0 + ew * 32 + r;
+                            if (mr < p.M) {
+                                uint4 v;
+                                lds128(tile + (uint32_t)(r * 128 + ((jq ^ (r & 7)) << 4)), v);
+                                *reinterpret_cast<uint4*>(static_cast<float*>(p.Y) + (size_t)mr * p.ldy + n0 + c0 + 4 * jq) = v;
                             }
                         }
                     }
