@@ -28,7 +28,7 @@ constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, EPI_WARP0 = 2, NUM_EPI_WARPS = 4;
 constexpr int NUM_THREADS = (EPI_WARP0 + NUM_EPI_WARPS) * 32;   // 192
 constexpr int TMEM_COLS = 512;
 
-struct __align__(8) Ctl {
+struct __align__(16) Ctl {
     uint64_t full[STAGES];
     uint64_t empty[STAGES];
     uint64_t tmem_full[2];
@@ -36,7 +36,8 @@ struct __align__(8) Ctl {
     uint32_t tmem_base;
     volatile int abort_flag;
 };
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + sizeof(Ctl);
+constexpr int EPI_TILE_BYTES = 32 * 32 * 4;         // one epilogue warp's 32 x 32 fp32 chunk, for the row/column trade
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + sizeof(Ctl) + NUM_EPI_WARPS * EPI_TILE_BYTES;
 
 constexpr uint32_t IDESC = umma_idesc_bf16(BM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
 
@@ -48,6 +49,7 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     unsigned char* sA = base;
     unsigned char* sB = base + STAGES * A_STAGE_BYTES;
     Ctl* ctl = reinterpret_cast<Ctl*>(sB + STAGES * B_STAGE_BYTES);
+    const uint32_t sEpi = smem_u32(reinterpret_cast<unsigned char*>(ctl) + sizeof(Ctl));   // NUM_EPI_WARPS x 4 KB
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_m = (M + BM - 1) / BM, tiles_n = (K + BN - 1) / BN;
@@ -144,25 +146,43 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                     uint32_t acc[32];
                     tc_ld32(tmem_base + ((uint32_t)(ew * 32) << 16) + (uint32_t)(buf * BN + c0), acc);
                     tc_wait_ld();
-                    if (m < M) {
-                        float* dst = Y + (size_t)m * K + n0 + c0;
-                        if (n0 + c0 + 32 <= K) {
+                    if (n0 + c0 + 32 <= K) {
+                        // A lane holds 32 consecutive outputs of its own row.  The warp trades rows for columns through
+                        // a 4 KB tile (chunk index XOR-ed with the row's low bits: conflict-free both ways) so that each
+                        // store writes four rows' whole 128-byte lines instead of half a sector of 32 rows.
+                        const uint32_t tile = sEpi + (uint32_t)(warp - EPI_WARP0) * EPI_TILE_BYTES;
+                        __syncwarp();
 #pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                reinterpret_cast<uint4*>(dst)[j] = make_uint4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+                        for (int j = 0; j < 8; ++j)
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(tile + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4))),
+                                         "r"(acc[4 * j]), "r"(acc[4 * j + 1]), "r"(acc[4 * j + 2]), "r"(acc[4 * j + 3]) : "memory");
+                        __syncwarp();
+                        const int rsub = lane >> 3, jq = lane & 7;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int r = 4 * i + rsub, mr = m0 + ew * 32 + r;
+                            if (mr < M) {
+                                uint4 v;
+                                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                                             : "r"(tile + (uint32_t)(r * 128 + ((jq ^ (r & 7)) << 4))) : "memory");
+                                *reinterpret_cast<uint4*>(Y + (size_t)mr * K + n0 + c0 + 4 * jq) = v;
+                            }
+                        }
+                        if (m < M) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) {
                                 asm("min.f32 %0, %0, %1, %2;" : "+f"(mn) : "f"(__uint_as_float(acc[j])), "f"(__uint_as_float(acc[j + 1])));
                                 asm("max.f32 %0, %0, %1, %2;" : "+f"(mx) : "f"(__uint_as_float(acc[j])), "f"(__uint_as_float(acc[j + 1])));
                             }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (n0 + c0 + j < K) {
-                                    const float v = __uint_as_float(acc[j]);
-                                    dst[j] = v; mn = fminf(mn, v); mx = fmaxf(mx, v);
-                                }
                         }
+                    } else if (m < M) {
+                        float* dst = Y + (size_t)m * K + n0 + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + c0 + j < K) {
+                                const float v = __uint_as_float(acc[j]);
+                                dst[j] = v; mn = fminf(mn, v); mx = fmaxf(mx, v);
+                            }
                     }
                 }
             }
