@@ -45,7 +45,7 @@ constexpr int BN = 256;                      // output channels per tile
 constexpr int BN_CTA = 128;                  // weight rows decoded per CTA
 constexpr int BK = 64;
 constexpr int STAGES = 4;                    // bf16 operand stages
-constexpr int CSTAGES = 6;                   // packed-code stages (small, so the TMA runs well ahead of the decode)
+constexpr int CSTAGES = 4;                   // packed-code stages (the TMA runs this many k-blocks ahead of the decode)
 constexpr int A_STAGE_BYTES = BM_CTA * BK * 2;      // 16 KB
 constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;      // 16 KB
 constexpr int AC_STAGE_BYTES = BM_CTA * BK;         // room for 8-bit codes (4-bit codes use half)
@@ -68,10 +68,11 @@ struct __align__(16) SharedCtl {
     alignas(16) float col[2][3][BN];   // per TMEM buffer: wsum, wscale, bias of the tile's columns (read as float4)
 };
 
-constexpr int EPI_TILE_BYTES = 32 * 32 * 4;         // one epilogue warp's 32 x 32 fp32 chunk, for the row/column trade
+constexpr int EPI_TILE_BYTES = 32 * 32 * 4;         // one epilogue warp's 32 x 32 fp32 chunk, staged for a TMA store
+constexpr int EPI_TILES = 2;                        // per epilogue warp: one being filled while the other is stored
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
-                              (size_t)CSTAGES * (AC_STAGE_BYTES + WC_STAGE_BYTES) + sizeof(SharedCtl) +
-                              (size_t)NUM_EPI_WARPS * EPI_TILE_BYTES;
+                              (size_t)NUM_EPI_WARPS * EPI_TILES * EPI_TILE_BYTES +
+                              (size_t)CSTAGES * (AC_STAGE_BYTES + WC_STAGE_BYTES) + sizeof(SharedCtl);
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 constexpr uint32_t IDESC = umma_idesc_bf16(2 * BM_CTA, BN, false, false);
@@ -224,15 +225,16 @@ struct Params {
 
 template <int A_BITS, int W_BITS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW) {
+qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                const __grid_constant__ CUtensorMap tmY) {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     unsigned char* sA = base;                                       // STAGES x 16 KB
     unsigned char* sB = sA + STAGES * A_STAGE_BYTES;                // STAGES x 16 KB
-    unsigned char* sAc = sB + STAGES * B_STAGE_BYTES;               // CSTAGES x 8 KB
+    unsigned char* sEpi = sB + STAGES * B_STAGE_BYTES;              // NUM_EPI_WARPS x EPI_TILES x 4 KB, 1024-byte aligned
+    unsigned char* sAc = sEpi + NUM_EPI_WARPS * EPI_TILES * EPI_TILE_BYTES;   // CSTAGES x 8 KB
     unsigned char* sWc = sAc + CSTAGES * AC_STAGE_BYTES;            // CSTAGES x 4 KB
     SharedCtl* ctl = reinterpret_cast<SharedCtl*>(sWc + CSTAGES * WC_STAGE_BYTES);
-    unsigned char* sEpi = reinterpret_cast<unsigned char*>(ctl) + sizeof(SharedCtl);   // NUM_EPI_WARPS x 4 KB
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                       // 0: issues the MMAs, 1: its peer
@@ -261,6 +263,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         mbar_init_fence();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmW);
+        tma_prefetch_desc(&tmY);
     }
     if (warp == MMA_WARP) tmem_alloc_pair(smem_u32(&ctl->tmem_base), TMEM_COLS);
     tc_fence_before();
@@ -468,7 +471,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         const int row = ew * 32 + lane;                            // accumulator row within the CTA
         const float zoff = (A_BITS == 8) ? 128.f : 8.f;            // the A operand is fed as q - 128 / q - 8
         const bool has_ws = p.wscale != nullptr, has_bias = p.bias != nullptr;
-        uint32_t t = 0;
+        uint32_t t = 0, nstore = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
             const int m0 = (tile % tiles_m) * 2 * BM_CTA + (int)rank * BM_CTA, n0 = (tile / tiles_m) * BN;
             const int buf = t & 1;
@@ -498,6 +501,8 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                     tc_ld32(tmem_base + ((uint32_t)(ew * 32) << 16) + (uint32_t)(buf * BN + c0), acc);
                     tc_wait_ld();
                     f32x2 yq[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) yq[j] = 0ull;
                     if (row_ok) {
                         // y = s_m * (acc + z_m * wsum_n) [* wscale_n] [+ bias_n], two columns per instruction
                         f32x2* y = yq;
@@ -552,40 +557,34 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                             }
                         }
                     }
-                    if (p.y_dtype == LRQ_F32 && n0 + c0 + 32 <= p.N) {
+                    if (p.y_dtype == LRQ_F32 && n0 + c0 + 32 <= p.N && m0 + ew * 32 < p.M) {     // warp-uniform; every store starts inside Y
                         // A lane holds 32 consecutive outputs of its own row; stored as they are, every store would
-                        // touch 32 different rows, half a sector each.  The warp trades rows for columns through a
-                        // 4 KB tile (16-byte chunk index XOR-ed with the row's low bits: conflict-free both ways), so
-                        // that each store writes four rows' whole 128-byte lines.
-                        const uint32_t tile = smem_u32(sEpi) + (uint32_t)ew * EPI_TILE_BYTES;
+                        // touch 32 different rows, half a sector each.  The warp lays its 32 x 32 chunk out in shared
+                        // memory (rows of 128 bytes, 128-byte swizzle: conflict-free) and one lane hands it to the TMA,
+                        // which writes whole lines, clips rows past M, and runs while the next chunk is prepared.
+                        const uint32_t tile = smem_u32(sEpi) + (uint32_t)((ew * EPI_TILES + (nstore & 1)) * EPI_TILE_BYTES);
+                        if (lane == 0) tma_store_wait_read<EPI_TILES - 1>();     // the store that last read this tile is done with it
                         __syncwarp();
-                        if (row_ok) {
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                float a, b, c2, d;
-                                unpack2(yq[2 * j], a, b); unpack2(yq[2 * j + 1], c2, d);
-                                sts128(tile + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4)), __float_as_uint(a), __float_as_uint(b),
-                                       __float_as_uint(c2), __float_as_uint(d));
-                            }
+                        for (int j = 0; j < 8; ++j) {
+                            float a, b, c2, d;
+                            unpack2(yq[2 * j], a, b); unpack2(yq[2 * j + 1], c2, d);
+                            sts128(tile + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4)), __float_as_uint(a), __float_as_uint(b),
+                                   __float_as_uint(c2), __float_as_uint(d));
                         }
+                        fence_async_smem();
                         __syncwarp();
-                        const int rsub = lane >> 3, jq = lane & 7;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const int r = 4 * i + rsub, mr = m0 + ew * 32 + r;
-                            if (mr < p.M) {
-                                uint4 v;
-                                lds128(tile + (uint32_t)(r * 128 + ((jq ^ (r & 7)) << 4)), v);
-                                *reinterpret_cast<uint4*>(static_cast<float*>(p.Y) + (size_t)mr * p.ldy + n0 + c0 + 4 * jq) = v;
-                            }
-                        }
+                        if (lane == 0) tma_store_2d(&tmY, n0 + c0, m0 + ew * 32, tile);
+                        ++nstore;
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(smem_u32(&ctl->tmem_empty[buf]), 0);
+            // CTA-scope release is enough: the accumulator reads above have completed (tcgen05.wait::ld)
+            if (lane == 0) mbar_arrive_cluster_light(smem_u32(&ctl->tmem_empty[buf]), 0);
         }
+        if (lane == 0) tma_store_wait_all();      // output tiles still in flight read this CTA's shared memory
     }
 
     // teardown: every role has left its loop.  Neither CTA may exit (or release TMEM) while its peer can
@@ -600,7 +599,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
 }
 
 template <int A_BITS, int W_BITS>
-lrq_status launch(const Params& p, const CUtensorMap& tmA, const CUtensorMap& tmW, int num_tiles, cudaStream_t st) {
+lrq_status launch(const Params& p, const CUtensorMap& tmA, const CUtensorMap& tmW, const CUtensorMap& tmY, int num_tiles, cudaStream_t st) {
     auto kern = qgemm_tc_kernel<A_BITS, W_BITS>;
     static int max_pairs = 0;                 // per process; the library targets identical GPUs
     cudaLaunchConfig_t cfg = {};
@@ -621,7 +620,7 @@ lrq_status launch(const Params& p, const CUtensorMap& tmA, const CUtensorMap& tm
     }
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
     cfg.gridDim = dim3(2 * pairs);
-    LRQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p, tmA, tmW));
+    LRQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p, tmA, tmW, tmY));
     return LRQ_OK;
 }
 
@@ -646,9 +645,12 @@ lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const
     CUtensorMap tmA, tmW;
     if (!lrq_tma::make_map_2d(&tmA, a_codes, 1, (uint64_t)M, a_row, a_row, BK * ab / 8, BM_CTA, false)) return LRQ_ERR_CUDA;
     if (!lrq_tma::make_map_2d(&tmW, L->codes, 1, (uint64_t)L->N, w_row, w_row, BK / 2, BN_CTA, false)) return LRQ_ERR_CUDA;
+    // fp32 outputs leave through TMA stores of 32 x 32 tiles; 16-bit outputs are stored directly (the map is then unused)
+    CUtensorMap tmY = tmW;
+    if (dt == LRQ_F32 && !lrq_tma::make_map_2d(&tmY, Y, 4, (uint64_t)M, (uint64_t)L->N, (uint64_t)ldy, 32, 32, true)) return LRQ_ERR_CUDA;
     const int tiles = ((M + 2 * BM_CTA - 1) / (2 * BM_CTA)) * ((L->N + BN - 1) / BN);
-    if (ab == 8 && L->w_bits == 4) return launch<8, 4>(p, tmA, tmW, tiles, st);
-    if (ab == 8) return launch<8, 3>(p, tmA, tmW, tiles, st);
-    if (ab == 4 && L->w_bits == 4) return launch<4, 4>(p, tmA, tmW, tiles, st);
-    return launch<4, 3>(p, tmA, tmW, tiles, st);
+    if (ab == 8 && L->w_bits == 4) return launch<8, 4>(p, tmA, tmW, tmY, tiles, st);
+    if (ab == 8) return launch<8, 3>(p, tmA, tmW, tmY, tiles, st);
+    if (ab == 4 && L->w_bits == 4) return launch<4, 4>(p, tmA, tmW, tmY, tiles, st);
+    return launch<4, 3>(p, tmA, tmW, tmY, tiles, st);
 }

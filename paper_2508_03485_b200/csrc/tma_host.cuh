@@ -24,7 +24,7 @@ inline EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Row-major matrix [rows, cols] of `elem_bytes`-byte elements (1: uint8, 2: bf16) with `ld` elements between
+// Row-major matrix [rows, cols] of `elem_bytes`-byte elements (1: uint8, 2: bf16, 4: fp32) with `ld` elements between
 // rows; tiles of box_cols x box_rows elements; out-of-range elements read as zero.  The base pointer and the
 // row pitch must be multiples of 16 bytes, box_cols * elem_bytes a multiple of 16 (and at most 128 with swizzle).
 inline bool make_map_2d(CUtensorMap* tm, const void* ptr, int elem_bytes, uint64_t rows, uint64_t cols, uint64_t ld,
@@ -35,7 +35,7 @@ inline bool make_map_2d(CUtensorMap* tm, const void* ptr, int elem_bytes, uint64
     const cuuint64_t strides[1] = {ld * (uint64_t)elem_bytes};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    return enc(tm, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+    return enc(tm, elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
                const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
