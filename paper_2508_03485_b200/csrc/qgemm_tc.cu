@@ -342,20 +342,31 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         const uint32_t sB0 = smem_u32(sB), sWc0 = smem_u32(sWc) + (uint32_t)row * (BK / 2);
         RingPos ring(grp);
         uint32_t it0 = 0;
-        bool ok = true;
+        bool ok = true, have_next = false;
+        float4 raw[NLEV / 4];
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, it0 += kblocks) {
             const int n_base = (tile / tiles_m) * BN + (int)rank * BN_CTA;
             const int n = min(n_base + row, p.N - 1);               // rows past N decode a valid table; never stored
             const float4* tab = reinterpret_cast<const float4*>(p.levels + (size_t)n * ngrp * NLEV);
             const int kb0 = (grp ^ (int)it0) & 1;
             Lut L;
-            float4 raw[NLEV / 4];
             // table index held in L / in raw, and the k-block at which the next table starts
             int gi = kb0 / kb_per_grp, fetched = gi, next_switch = (gi + 1) * kb_per_grp;
             if (kb0 < kblocks) {
+                if (!(ngrp == 1 && have_next)) {                    // per-channel tables arrive a tile ahead (below)
 #pragma unroll
-                for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)gi * (NLEV / 4) + j);
+                    for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tab + (size_t)gi * (NLEV / 4) + j);
+                }
                 build_lut<W_BITS>(L, raw);
+            }
+            have_next = false;
+            if (ngrp == 1 && tile + num_pairs < num_tiles) {
+                // per-channel tables: the next tile's table is fetched now, a whole tile before it is needed
+                const int nn = min(((tile + num_pairs) / tiles_m) * BN + (int)rank * BN_CTA + row, p.N - 1);
+                const float4* tn = reinterpret_cast<const float4*>(p.levels + (size_t)nn * NLEV);
+#pragma unroll
+                for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tn + j);
+                have_next = true;
             }
             for (int kb = kb0; kb < kblocks; kb += 2) {
                 if (ngrp > 1) {                                     // grouped tables: switch, and fetch one step ahead
