@@ -15,7 +15,8 @@
  * no pin can reach (they are choices, not consequences) are "parity unpinned": the merge of
  * the two zero codes into one table entry, the clipping grid values, the search objective,
  * the block-diagonal Hadamard for sizes that are not a power of two, and the symmetric
- * activation mode.
+ * activation mode.  The smoothing vector of orc_smooth (Sec. 5.1) is an input here: how it is
+ * calibrated (migration strength 0.5) is outside the path, so only its application is pinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -333,4 +334,33 @@ int orc_dequantize_act(const int32_t *Q, const double *S, const int32_t *Z, int 
         for (int k = 0; k < K; ++k)
             Xf[(size_t)m * K + k] = S[m] * ((double)Q[(size_t)m * K + k] + (double)Z[m]);
     return 0;
+}
+
+
+/* ------------------------------------------------------------------------------------------
+ * Sec. 5.1 (smoothing, after SmoothQuant): activations are divided channel-wise by a smoothing
+ * factor that the weights absorb, X' = X diag(p), W' = W diag(1/p), so that X' W'^T = X W^T.
+ * p (length K) holds the multipliers 1/lambda_k applied to the activations.  Y = X diag(p).
+ * ---------------------------------------------------------------------------------------- */
+int orc_smooth(const double *X, int M, int K, const double *p, double *Y) {
+    if (M <= 0 || K <= 0) return -1;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m)
+        for (int k = 0; k < K; ++k) Y[(size_t)m * K + k] = X[(size_t)m * K + k] * p[k];
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Sec. 4.2, Eq. 11: fluctuation metric of a layer's activations X (B x N x C values, here a
+ * matrix of M = B*N tokens by K = C channels):  J = ||X||_F / sqrt(B N C).
+ * Eq. 12: the layer takes the Hadamard rotation when J < Thr, the outlier-aware one otherwise.
+ * Returns J; *kind gets 1 (Hadamard) or 2 (outlier-aware dense rotation).
+ * ---------------------------------------------------------------------------------------- */
+double orc_fluctuation_metric(const double *X, int M, int K, double thr, int *kind) {
+    double ss = 0.0;
+    for (int m = 0; m < M; ++m)
+        for (int k = 0; k < K; ++k) ss += X[(size_t)m * K + k] * X[(size_t)m * K + k];
+    const double J = sqrt(ss) / sqrt((double)M * (double)K);
+    if (kind) *kind = J < thr ? 1 : 2;
+    return J;
 }

@@ -21,7 +21,7 @@ _LIB = os.path.join(_HERE, "liblrq_oracle.so")
 __all__ = [
     "build", "num_threads", "hadamard_matrix", "rotate_hadamard_explicit", "rotate_hadamard_fwht",
     "rotate_dense", "quantize_act", "dequantize_act", "level_value", "tlq_quantize", "qmatmul",
-    "TLQResult", "qlinear",
+    "TLQResult", "qlinear", "smooth", "fluctuation_metric",
 ]
 
 
@@ -45,6 +45,8 @@ def _L():
         _lib = ctypes.CDLL(build())
         _lib.orc_level_value.restype = ctypes.c_double
         _lib.orc_level_value.argtypes = [ctypes.c_double, ctypes.c_int]
+        _lib.orc_fluctuation_metric.restype = ctypes.c_double
+        _lib.orc_fluctuation_metric.argtypes = [_dp, ctypes.c_int, ctypes.c_int, ctypes.c_double, _ip]
     return _lib
 
 
@@ -95,6 +97,27 @@ def rotate_dense(X, R):
     Y = np.empty_like(X)
     _L().orc_rotate_dense(xp, M, K, rp, Y.ctypes.data_as(_dp))
     return Y
+
+
+def smooth(X, p):
+    """X diag(p): the channel-wise smoothing multipliers applied to the activations (Sec. 5.1)."""
+    X, xp = _d(X)
+    p, pp = _d(p)
+    M, K = X.shape
+    assert p.shape == (K,)
+    Y = np.empty_like(X)
+    _L().orc_smooth(xp, M, K, pp, Y.ctypes.data_as(_dp))
+    return Y
+
+
+def fluctuation_metric(X, thr: float = 1.0):
+    """J = ||X||_F / sqrt(B N C) (Sec. 4.2, Eq. 11) and the rotation kind Eq. 12 picks:
+    1 = Hadamard (J < thr), 2 = outlier-aware dense rotation.  Returns (J, kind)."""
+    X, xp = _d(X)
+    M, K = X.shape
+    kind = ctypes.c_int32(0)
+    J = _L().orc_fluctuation_metric(xp, M, K, float(thr), ctypes.byref(kind))
+    return float(J), int(kind.value)
 
 
 def quantize_act(Y, bits: int, mode: int = 0):
@@ -185,9 +208,11 @@ def qmatmul(Q, S, Z, tlq: TLQResult, wscale=None, bias=None):
 
 
 def qlinear(X, tlq: TLQResult, a_bits: int, rot: str, had_block: int = 0, R=None, mode: int = 0,
-            wscale=None, bias=None):
-    """The whole layer on already-widened inputs: rotate (Eq. 12) -> per-token quantize (Eq. 1) ->
-    contraction with the TLQ table and epilogue (Eq. 10).  Returns (Y, codes, s, z)."""
+            wscale=None, bias=None, prescale=None):
+    """The whole layer on already-widened inputs: [smooth (Sec. 5.1) ->] rotate (Eq. 12) -> per-token
+    quantize (Eq. 1) -> contraction with the TLQ table and epilogue (Eq. 10).  Returns (Y, codes, s, z)."""
+    if prescale is not None:
+        X = smooth(X, prescale)
     if rot == "hadamard":
         Yr = rotate_hadamard_fwht(X, had_block)
     elif rot == "dense":
