@@ -98,6 +98,10 @@ typedef struct {
     const void* R_bf16;      /* dev bf16 [K,K] row-major for DENSE (y_i = sum_l x_l R[l,i])        */
     int a_bits;              /* 4 or 8                                                            */
     lrq_act_mode mode;
+    const float* prescale;   /* nullable dev float [K], 16-byte aligned: smoothing multipliers applied
+                                channel-wise before the rotation (Sec. 5.1: X' = X diag(prescale), the
+                                weights having absorbed diag(1/prescale)).  HADAMARD / NONE only; for a
+                                DENSE rotation fold diag(prescale) into R.                            */
 } lrq_act_params;
 
 /* Bytes of workspace lrq_rotate_quantize_act needs for M tokens (0 unless kind == DENSE). */
@@ -113,6 +117,17 @@ size_t lrq_act_workspace_bytes(int M, int K, const lrq_act_params* p);
 lrq_status lrq_rotate_quantize_act(const void* X_bf16, int M, int K, long ldx, const lrq_act_params* p,
                                    uint8_t* a_codes, float* a_scale, int32_t* a_zp,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Adaptive Rotation Scheme, the per-layer choice (Sec. 4.2): fluctuation metric of a batch of
+ * calibration activations, J = ||X||_F / sqrt(M K) (Eq. 11), and the rotation kind of Eq. 12:
+ * LRQ_ROT_HADAMARD when J < threshold (the paper uses 1), LRQ_ROT_DENSE otherwise.
+ *   X         dev bf16 [M,ldx], 32-byte aligned, K and ldx multiples of 16
+ *   J, kind   dev float / int32, one element each (out)
+ *   workspace dev, 8 bytes, 8-byte aligned (one double; cleared by the call)
+ * ------------------------------------------------------------------------------------------- */
+lrq_status lrq_ars_select(const void* X_bf16, int M, int K, long ldx, double threshold, float* J, int32_t* kind,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
  * lrq_rotate_quantize_act for callers that cannot hand over device scratch.

@@ -20,7 +20,7 @@ _TORCH_DT = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16}
 EXPORTS = [
     "lrq_tlq_quantize_weights", "lrq_act_workspace_bytes", "lrq_rotate_quantize_act", "lrq_layer_create",
     "lrq_layer_destroy", "lrq_workspace_bytes", "lrq_qlinear", "lrq_qlinear_stack", "lrq_qgemm_codes",
-    "lrq_device_status", "lrq_status_string", "lrq_version", "lrq_rotate_quantize_act_static",
+    "lrq_device_status", "lrq_status_string", "lrq_version", "lrq_rotate_quantize_act_static", "lrq_ars_select",
 ]
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -40,7 +40,7 @@ class _TlqParams(C.Structure):
 
 class _ActParams(C.Structure):
     _fields_ = [("kind", C.c_int), ("had_block", C.c_int), ("R_bf16", C.c_void_p),
-                ("a_bits", C.c_int), ("mode", C.c_int)]
+                ("a_bits", C.c_int), ("mode", C.c_int), ("prescale", C.c_void_p)]
 
 
 _lib = None
@@ -71,6 +71,7 @@ def load_library() -> C.CDLL:
     lib.lrq_qlinear_stack.argtypes = [C.POINTER(vp), ci, C.POINTER(vp), C.POINTER(ci), C.POINTER(cl),
                                       C.POINTER(vp), ci, C.POINTER(cl), vp, sz, vp]
     lib.lrq_qgemm_codes.argtypes = [vp, vp, vp, vp, ci, vp, ci, cl, ci, vp]
+    lib.lrq_ars_select.argtypes = [vp, ci, ci, cl, C.c_double, vp, vp, vp, sz, vp]
     lib.lrq_device_status.argtypes = [vp]
     lib.lrq_status_string.argtypes = [ci]
     lib.lrq_status_string.restype = C.c_char_p
@@ -143,20 +144,40 @@ def lrq_tlq_quantize_weights(W_rot: torch.Tensor, w_bits: int, group_size: int =
     return TLQWeights(codes, levels, meta, wsum, int(w_bits), int(group_size))
 
 
-def _act_params(kind: int, had_block: int, R: Optional[torch.Tensor], a_bits: int, mode: int) -> _ActParams:
-    return _ActParams(int(kind), int(had_block), 0 if R is None else R.data_ptr(), int(a_bits), int(mode))
+def _act_params(kind: int, had_block: int, R: Optional[torch.Tensor], a_bits: int, mode: int,
+                prescale: Optional[torch.Tensor] = None) -> _ActParams:
+    if prescale is not None:
+        assert prescale.dtype == torch.float32 and prescale.is_contiguous()
+    return _ActParams(int(kind), int(had_block), 0 if R is None else R.data_ptr(), int(a_bits), int(mode),
+                      0 if prescale is None else prescale.data_ptr())
+
+
+def lrq_ars_select(X: torch.Tensor, threshold: float = 1.0, stream=None):
+    """Fluctuation metric J of calibration activations and the rotation kind it selects (Eqs. 11-12).
+    Returns (J float32[1], kind int32[1]) device tensors."""
+    _need_cuda(X)
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M, K = X.shape
+    J = torch.empty(1, dtype=torch.float32, device=X.device)
+    kind = torch.empty(1, dtype=torch.int32, device=X.device)
+    ws = torch.empty(1, dtype=torch.float64, device=X.device)
+    rc = load_library().lrq_ars_select(_ptr(X), M, K, X.stride(0), float(threshold), _ptr(J), _ptr(kind), _ptr(ws), 8,
+                                       _stream(stream))
+    _check(rc, "lrq_ars_select")
+    return J, kind
 
 
 def lrq_rotate_quantize_act(X: torch.Tensor, kind: int, a_bits: int, had_block: int = 0,
                             R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM,
-                            workspace: Optional[torch.Tensor] = None, stream=None, out=None):
+                            workspace: Optional[torch.Tensor] = None, stream=None, out=None,
+                            prescale: Optional[torch.Tensor] = None):
     """Rotation + per-token quantization (Eq. 12, Eq. 1) of device bf16 [M,K] activations.
     Returns (codes uint8, scale float32 [M], zero_point int32 [M])."""
-    _need_cuda(X, R, workspace)
+    _need_cuda(X, R, workspace, prescale)
     assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
     M, K = X.shape
     lib = load_library()
-    p = _act_params(kind, had_block, R, a_bits, mode)
+    p = _act_params(kind, had_block, R, a_bits, mode, prescale)
     need = int(lib.lrq_act_workspace_bytes(M, K, C.byref(p)))
     if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
         workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
@@ -203,11 +224,13 @@ class QLayer:
 
     def __init__(self, tlq: TLQWeights, N: int, K: int, kind: int, a_bits: int, had_block: int = 0,
                  R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM,
-                 wscale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None):
-        _need_cuda(tlq.codes, tlq.levels, tlq.wsum, R, wscale, bias)
+                 wscale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                 prescale: Optional[torch.Tensor] = None):
+        _need_cuda(tlq.codes, tlq.levels, tlq.wsum, R, wscale, bias, prescale)
+        self.prescale = prescale
         self.tlq, self.N, self.K, self.R, self.wscale, self.bias = tlq, N, K, R, wscale, bias
         self.kind, self.a_bits, self.had_block, self.mode = kind, a_bits, had_block, mode
-        self._p = _act_params(kind, had_block, R, a_bits, mode)
+        self._p = _act_params(kind, had_block, R, a_bits, mode, prescale)
         h = C.c_void_p()
         rc = load_library().lrq_layer_create(C.byref(h), N, K, tlq.w_bits, tlq.group, _ptr(tlq.codes),
                                              _ptr(tlq.levels), _ptr(tlq.wsum), _ptr(wscale), _ptr(bias),

@@ -32,9 +32,11 @@ static lrq_status check_act(const lrq_act_params* p, int K) {
         case LRQ_ROT_DENSE:
             if (!p->R_bf16) return LRQ_ERR_INVALID_ARG;
             if (!lrq_aligned(p->R_bf16, 16)) return LRQ_ERR_INVALID_ARG;
+            if (p->prescale) return LRQ_ERR_UNSUPPORTED;      // fold diag(prescale) into R instead
             break;
         default: return LRQ_ERR_INVALID_ARG;
     }
+    if (p->prescale && !lrq_aligned(p->prescale, 16)) return LRQ_ERR_INVALID_ARG;
     return LRQ_OK;
 }
 
@@ -65,7 +67,7 @@ extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long 
         return lrq_launch_quantize_f32(Yr, M, K, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
     }
     const int B = p->kind == LRQ_ROT_HADAMARD ? p->had_block : 1;
-    return lrq_launch_rotq_hadamard(X, M, K, ldx, B, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
+    return lrq_launch_rotq_hadamard(X, M, K, ldx, B, p->a_bits, p->mode, p->prescale, a_codes, a_scale, a_zp, stream);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -106,6 +108,15 @@ extern "C" lrq_status lrq_rotate_quantize_act_static(const void* X, int M, int K
     if (!scratch) return LRQ_ERR_CUDA;
     return lrq_rotate_quantize_act(X, M, K, ldx, p, a_codes, a_scale, a_zp, scratch, LRQ_STATIC_SCRATCH_BYTES,
                                    cuda_stream);
+}
+
+extern "C" lrq_status lrq_ars_select(const void* X, int M, int K, long ldx, double threshold, float* J, int32_t* kind,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!X || !J || !kind || M <= 0 || K <= 0) return LRQ_ERR_INVALID_ARG;
+    if (K % 16 || ldx < K || ldx % 16 || !lrq_aligned(X, 32)) return LRQ_ERR_UNSUPPORTED;   // 256-bit loads
+    if (!workspace || workspace_bytes < sizeof(double) || !lrq_aligned(workspace, 8)) return LRQ_ERR_WORKSPACE;
+    return lrq_launch_ars_metric(X, M, K, ldx, threshold, J, reinterpret_cast<int*>(kind), static_cast<double*>(workspace),
+                                 (cudaStream_t)cuda_stream);
 }
 
 extern "C" lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size,

@@ -30,7 +30,7 @@ struct lrq_layer {
 int* lrq_status_word();               // device address of the word (allocated lazily, once per process)
 
 // rotq.cu
-lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B, int a_bits, int mode,
+lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B, int a_bits, int mode, const float* prescale,
                                     uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
 lrq_status lrq_launch_quantize_f32(const float* Y, int M, int K, long ldy, int a_bits, int mode,
                                    uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
@@ -42,6 +42,10 @@ lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void*
 // scale / zero-point outputs: each row's extremes are read before its results are written).
 lrq_status lrq_launch_quantize_f32_ext(const float* Y, int M, int K, int a_bits, int mode, uint8_t* codes,
                                        float* scale, int32_t* zp, cudaStream_t st);
+
+// rotq.cu : fluctuation metric J (Eq. 11) and the kind Eq. 12 picks; acc is one double of device scratch
+lrq_status lrq_launch_ars_metric(const void* X, int M, int K, long ldx, double thr, float* J, int* kind, double* acc,
+                                 cudaStream_t st);
 
 #ifdef __CUDACC__
 // Order-preserving map between fp32 and int32 (and back), so that integer min/max reductions serve floats.

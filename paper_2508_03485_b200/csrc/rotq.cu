@@ -65,6 +65,7 @@ __device__ __forceinline__ int quant1(float u, const TokenQ& t, int qmax) {
 template <bool SRC_F32>
 __global__ void __launch_bounds__(256)
 rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log2B, int a_bits, int mode,
+                    const float* __restrict__ prescale,
                     uint8_t* __restrict__ codes, float* __restrict__ scale, int32_t* __restrict__ zp) {
     extern __shared__ float row[];
     __shared__ float red_mn[8], red_mx[8], red_am[8];
@@ -81,6 +82,10 @@ rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log
         for (int c = tid; c < nchunk; c += nthr) {
             float v[8];
             unpack_bf16x8(src[c], v);
+            if (prescale) {                                   // smoothing multipliers (Sec. 5.1), before the rotation
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] *= __ldg(prescale + c * 8 + i);
+            }
             if (log2B >= 3) bfly8(v);
 #pragma unroll
             for (int i = 0; i < 8; ++i) row[c * 8 + i] = v[i];
@@ -169,6 +174,7 @@ __device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64
 __device__ __forceinline__ void unpack2(f32x2 r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
 __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
 __device__ __forceinline__ float min3(float a, float b, float c) { float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
 __device__ __forceinline__ float max3(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
@@ -246,6 +252,7 @@ __device__ __forceinline__ TokenQ token_params_fast(float mn, float mx, int a_bi
 template <int LOG2B, int A_BITS, int MAX_THREADS, int MIN_CTAS, bool WIDE>
 __global__ void __launch_bounds__(MAX_THREADS, MIN_CTAS)
 rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, int mode, int tok_per_cta, int num_groups,
+                 const float* __restrict__ prescale,
                  uint8_t* __restrict__ codes, float* __restrict__ scale, int32_t* __restrict__ zp) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr int NP = EPT / 2;                      // element pairs per thread
@@ -282,6 +289,14 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
 #pragma unroll
             for (int c = 0; c < 4; ++c)
                 P[4 * i + c] = pack2(__uint_as_float(w[c] << 16), __uint_as_float(w[c] & 0xffff0000u));
+        }
+        if (prescale) {                                       // smoothing multipliers (Sec. 5.1), before the rotation
+            const float4* ps = reinterpret_cast<const float4*>(prescale + (size_t)j * EPT);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 f = __ldg(ps + i);
+                P[2 * i] = mul2(P[2 * i], pack2(f.x, f.y)); P[2 * i + 1] = mul2(P[2 * i + 1], pack2(f.z, f.w));
+            }
         }
         // the next group's loads fly while this group is transformed
         {
@@ -462,7 +477,69 @@ lrq_status lrq_launch_quantize_f32_ext(const float* Y, int M, int K, int a_bits,
     return LRQ_OK;
 }
 
-static lrq_status launch_generic(bool f32, const void* X, int M, int K, long ldx, int log2B, int a_bits, int mode,
+// ------------------------------------------------------------------------------------------------
+// Fluctuation metric of a layer's activations (Sec. 4.2, Eq. 11): J = ||X||_F / sqrt(M K), and the rotation
+// kind the threshold rule of Eq. 12 picks.  HBM-bound: 2 bytes per element, read once with 256-bit loads.
+// Squares of bf16 values are exact in fp32; a thread sums its 16 squares in fp32 (relative error below
+// 16 * 2^-24), everything above that in fp64.
+// ------------------------------------------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(256)
+sumsq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, double* __restrict__ acc) {
+    const int cpr = K >> 4;                                  // 32-byte chunks per row
+    const long total = (long)M * cpr;
+    double part = 0.0;
+    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+        const long m = i / cpr;
+        const int c = (int)(i - m * cpr);
+        uint32_t r[8];
+        asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                     : "l"(X + m * ldx + 16 * c));
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float lo = __uint_as_float(r[k] << 16), hi = __uint_as_float(r[k] & 0xffff0000u);
+            s = fmaf(lo, lo, s); s = fmaf(hi, hi, s);
+        }
+        part += (double)s;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    __shared__ double wsum[8];
+    if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = part;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < 8; ++w) t += wsum[w];
+        atomicAdd(acc, t);
+    }
+}
+__global__ void ars_finish_kernel(const double* __restrict__ acc, double count, double thr, float* __restrict__ J,
+                                  int* __restrict__ kind) {
+    const double j = sqrt(*acc) / sqrt(count);
+    *J = (float)j;
+    *kind = j < thr ? (int)LRQ_ROT_HADAMARD : (int)LRQ_ROT_DENSE;
+}
+}  // namespace
+
+lrq_status lrq_launch_ars_metric(const void* X, int M, int K, long ldx, double thr, float* J, int* kind, double* acc,
+                                 cudaStream_t st) {
+    int dev = 0, sms = 0;
+    LRQ_CUDA_TRY(cudaGetDevice(&dev));
+    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    LRQ_CUDA_TRY(cudaMemsetAsync(acc, 0, sizeof(double), st));
+    const long total = (long)M * (K >> 4);
+    long blocks = (total + 255) / 256;
+    if (blocks > (long)sms * 8) blocks = (long)sms * 8;
+    sumsq_kernel<<<(int)blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx, acc);
+    LRQ_CUDA_TRY(cudaGetLastError());
+    ars_finish_kernel<<<1, 1, 0, st>>>(acc, (double)M * (double)K, thr, J, kind);
+    LRQ_CUDA_TRY(cudaGetLastError());
+    return LRQ_OK;
+}
+
+static lrq_status launch_generic(bool f32, const void* X, int M, int K, long ldx, int log2B, int a_bits, int mode, const float* prescale,
                                  uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st) {
     const size_t smem = (size_t)K * sizeof(float);
     if (smem > 200 * 1024) return LRQ_ERR_UNSUPPORTED;
@@ -470,13 +547,13 @@ static lrq_status launch_generic(bool f32, const void* X, int M, int K, long ldx
     if (smem > 40 * 1024)
         LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int threads = (K >= 2048) ? 256 : (K >= 1024 ? 128 : 64);
-    kern<<<M, threads, smem, st>>>(X, M, K, ldx, log2B, a_bits, mode, codes, scale, zp);
+    kern<<<M, threads, smem, st>>>(X, M, K, ldx, log2B, a_bits, mode, prescale, codes, scale, zp);
     LRQ_CUDA_TRY(cudaGetLastError());
     return LRQ_OK;
 }
 
 template <int LOG2B>
-static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits, int mode, uint8_t* codes,
+static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits, int mode, const float* prescale, uint8_t* codes,
                               float* scale, int32_t* zp, cudaStream_t st) {
     const int tpt = K / EPT;
     // whole tokens per CTA: thread count a multiple of 32, at least 256 when the token is small
@@ -489,7 +566,7 @@ static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits,
     size_t smem = 3 * 2 * sizeof(int) * T + 16;
     if (LOG2B > 10) smem += (size_t)threads * EPT * sizeof(float);
     // register budget by CTA size: three CTAs of up to 288 threads, two of up to 384, else one
-    typedef void (*Kern)(const __nv_bfloat16*, int, int, long, int, int, int, uint8_t*, float*, int32_t*);
+    typedef void (*Kern)(const __nv_bfloat16*, int, int, long, int, int, int, const float*, uint8_t*, float*, int32_t*);
     // 256-bit accesses when every thread's 64 input bytes and 32 code bytes start on 32-byte boundaries
     const bool wide = lrq_aligned(X, 32) && (ldx % 16) == 0 && lrq_aligned(codes, 32);
     Kern kern;
@@ -508,12 +585,12 @@ static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits,
     if (per_sm < 1) return LRQ_ERR_UNSUPPORTED;
     const int groups = (M + T - 1) / T;
     const int grid = groups < sms * per_sm ? groups : sms * per_sm;
-    kern<<<grid, threads, smem, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx, mode, T, groups, codes, scale, zp);
+    kern<<<grid, threads, smem, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx, mode, T, groups, prescale, codes, scale, zp);
     LRQ_CUDA_TRY(cudaGetLastError());
     return LRQ_OK;
 }
 
-lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B, int a_bits, int mode,
+lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B, int a_bits, int mode, const float* prescale,
                                     uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st) {
     int log2B = 0;
     while ((1 << log2B) < B) ++log2B;
@@ -522,7 +599,7 @@ lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B
     if (fast_ok) {
         lrq_status r = LRQ_ERR_UNSUPPORTED;
         switch (log2B) {
-#define LRQ_CASE(L) case L: r = launch_fast<L>(X, M, K, ldx, a_bits, mode, codes, scale, zp, st); break;
+#define LRQ_CASE(L) case L: r = launch_fast<L>(X, M, K, ldx, a_bits, mode, prescale, codes, scale, zp, st); break;
             LRQ_CASE(3) LRQ_CASE(4) LRQ_CASE(5) LRQ_CASE(6) LRQ_CASE(7) LRQ_CASE(8) LRQ_CASE(9) LRQ_CASE(10)
             LRQ_CASE(11) LRQ_CASE(12)
 #undef LRQ_CASE
@@ -530,10 +607,10 @@ lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B
         }
         if (r != LRQ_ERR_UNSUPPORTED) return r;
     }
-    return launch_generic(false, X, M, K, ldx, log2B, a_bits, mode, codes, scale, zp, st);
+    return launch_generic(false, X, M, K, ldx, log2B, a_bits, mode, prescale, codes, scale, zp, st);
 }
 
 lrq_status lrq_launch_quantize_f32(const float* Y, int M, int K, long ldy, int a_bits, int mode,
                                    uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st) {
-    return launch_generic(true, Y, M, K, ldy, 0, a_bits, mode, codes, scale, zp, st);
+    return launch_generic(true, Y, M, K, ldy, 0, a_bits, mode, nullptr, codes, scale, zp, st);
 }

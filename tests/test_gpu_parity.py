@@ -243,3 +243,36 @@ def test_qlinear_stack_replays_from_a_cuda_graph(P):
         for layer, X, Y in zip(layers, Xs, Ys):
             assert torch.equal(Y, P.lrq_qlinear(layer, X, P.F32))
     assert P.lrq_device_status() == 0
+
+
+# --------------------------------------------------------------------------------- smoothing, ARS metric
+@pytest.mark.parametrize("M,K,B,a_bits", [(40, 1152, 128, 8), (33, 1536, 512, 4), (9, 72, 8, 8), (5, 6144, 2048, 4)])
+def test_rotate_quantize_with_smoothing(P, orc, M, K, B, a_bits):
+    # Sec. 5.1: channel-wise multipliers applied before the rotation (fast and generic kernels)
+    xb = make_activations(300 + K, M, K, n_salient=8, salient_x=60.0)
+    rng = np.random.default_rng(K)
+    p = (1.0 / np.sqrt(np.abs(bf16_bits_to_f64(xb)).max(axis=0) + 1e-3) * rng.uniform(0.8, 1.25, K)).astype(np.float32)
+    q, s, z = P.lrq_rotate_quantize_act(PU.bf16_to_device(xb), P.ROT_HADAMARD, a_bits, B,
+                                        prescale=torch.from_numpy(p).cuda())
+    Yr = orc.rotate_hadamard_fwht(orc.smooth(bf16_bits_to_f64(xb), p.astype(np.float64)), B)
+    oq, os_, oz = orc.quantize_act(Yr, a_bits)
+    PU.check_act(PU.act_codes_to_numpy(q, a_bits), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, f"smooth {M}x{K}")
+
+
+def test_smoothing_is_refused_for_a_dense_rotation(P):
+    X = torch.zeros((8, 128), dtype=torch.bfloat16, device="cuda")
+    R = torch.zeros((128, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(P.LrqError) as e:
+        P.lrq_rotate_quantize_act(X, P.ROT_DENSE, 8, R=R, prescale=torch.ones(128, device="cuda"))
+    assert e.value.code == 2
+
+
+@pytest.mark.parametrize("M,K,n_sal,thr", [(256, 1152, 0, 1.0), (300, 1536, 16, 1.0), (4096, 4608, 0, 1.0), (17, 64, 2, 5.0)])
+def test_ars_metric_and_choice(P, orc, M, K, n_sal, thr):
+    # Eq. 11 / Eq. 12 against the oracle; tolerance 1e-6: squares of bf16 are exact in fp32 and at most 16 of them
+    # are summed in fp32 (relative error below 16 * 2^-24) before everything goes on in fp64
+    xb = make_activations(400 + K, M, K, n_salient=n_sal, salient_x=100.0)
+    J, kind = P.lrq_ars_select(PU.bf16_to_device(xb), thr)
+    Jo, ko = orc.fluctuation_metric(bf16_bits_to_f64(xb), thr)
+    assert abs(J.item() - Jo) <= 1e-6 * Jo
+    assert abs(Jo - thr) > 1e-4 * thr and kind.item() == ko
