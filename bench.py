@@ -37,9 +37,9 @@ from lrq_workloads import bf16_bits_to_f64, config_layers, default_clip_grid  # 
 # profiles/, keyed by the kernel and layer the roofline object describes.  A key is dropped (traffic: null) when its
 # kernel changes after the capture.
 NCU_TRAFFIC_BYTES = {
-    "qgemm cfg1 fc1": 7.83e6 + 23.37e6,
-    "qgemm cfg3 fc1": 27.03e6 + 174.04e6,
-    "qgemm cfg4 b0.fc1": 123.76e6 + 552.45e6,
+    "qgemm cfg1 fc1": 7.77e6 + 19.13e6,
+    "qgemm cfg3 fc1": 27.39e6 + 169.47e6,
+    "qgemm cfg4 b0.fc1": 220.77e6 + 555.42e6,
     "rotq cfg1 fc2": None,                      # 57 MB case not captured; the M = 32768 capture of the same layer shape:
     "rotq cfg4 b0.fc2": 302.28e6 + 123.51e6,
     "rotq cfg3 fc2": 113.83e6 + 16.29e6,
@@ -403,13 +403,16 @@ def run_kernel(args):
     elif args.kernel == "qgemm":
         fn = lambda: P.lrq_qgemm_codes(L, rq[0], rq[1], rq[2], P.F32, args.gemm_impl, Y, stream)
         units, unit = 2.0 * M * s.N * s.K / 1e12, "TFLOP/s"
+    elif args.kernel == "ars":
+        fn = lambda: P.lrq_ars_select(X, 1.0, stream)
+        units, unit = M * 2.0 * s.K / 1e9, "GB/s"
     else:
         fn = lambda: P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid)
         units, unit = s.N * s.K / 1e9, "Gweights/s"
     for _ in range(max(1, args.warmup)):
         fn()
     torch.cuda.synchronize()
-    if not args.no_graph and args.kernel != "tlq":
+    if not args.no_graph and args.kernel in ("rotq", "qgemm"):
         call = fn
         if args.kernel == "rotq":
             call = lambda: P.lrq_rotate_quantize_act(X, kind, s.a_bits, s.had_block, R, workspace=ws, out=rq)
@@ -444,7 +447,7 @@ def main():
     ap.add_argument("--gemm-impl", type=int, default=0, choices=[0, 1],
                     help="kernel timed alone for the roofline object: 0 tcgen05, 1 CUDA-core baseline")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph replay of the step")
-    ap.add_argument("--kernel", default=None, choices=["rotq", "qgemm", "tlq"], help="time one kernel only")
+    ap.add_argument("--kernel", default=None, choices=["rotq", "qgemm", "tlq", "ars"], help="time one kernel only")
     ap.add_argument("--layer", type=int, default=0, help="layer index of the workload for --kernel")
     ap.add_argument("--tokens", type=int, default=0, help="override M for --kernel")
     args = ap.parse_args()

@@ -487,22 +487,37 @@ namespace {
 __global__ void __launch_bounds__(256)
 sumsq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, double* __restrict__ acc) {
     const int cpr = K >> 4;                                  // 32-byte chunks per row
-    const long total = (long)M * cpr;
     double part = 0.0;
-    for (long i = blockIdx.x * (long)blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
-        const long m = i / cpr;
-        const int c = (int)(i - m * cpr);
-        uint32_t r[8];
-        asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                     : "l"(X + m * ldx + 16 * c));
-        float s = 0.f;
+    // a warp walks over rows (grid stride), its lanes over the row's chunks, four loads in flight per lane
+    const int lane = threadIdx.x & 31;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (int m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; m < M; m += nwarps) {
+        const __nv_bfloat16* row = X + (size_t)m * ldx;
+        for (int c0 = lane; c0 < cpr; c0 += 128) {
+            uint32_t r[4][8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const float lo = __uint_as_float(r[k] << 16), hi = __uint_as_float(r[k] & 0xffff0000u);
-            s = fmaf(lo, lo, s); s = fmaf(hi, hi, s);
+            for (int u = 0; u < 4; ++u) {
+                const int c = c0 + 32 * u;
+                if (c < cpr)
+                    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                                 : "=r"(r[u][0]), "=r"(r[u][1]), "=r"(r[u][2]), "=r"(r[u][3]), "=r"(r[u][4]), "=r"(r[u][5]),
+                                   "=r"(r[u][6]), "=r"(r[u][7]) : "l"(row + 16 * c));
+                else {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) r[u][k] = 0;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float s = 0.f;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float lo = __uint_as_float(r[u][k] << 16), hi = __uint_as_float(r[u][k] & 0xffff0000u);
+                    s = fmaf(lo, lo, s); s = fmaf(hi, hi, s);
+                }
+                part += (double)s;
+            }
         }
-        part += (double)s;
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
@@ -529,8 +544,7 @@ lrq_status lrq_launch_ars_metric(const void* X, int M, int K, long ldx, double t
     LRQ_CUDA_TRY(cudaGetDevice(&dev));
     LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     LRQ_CUDA_TRY(cudaMemsetAsync(acc, 0, sizeof(double), st));
-    const long total = (long)M * (K >> 4);
-    long blocks = (total + 255) / 256;
+    long blocks = ((long)M + 7) / 8;                         // 8 warps per CTA, one row per warp and step
     if (blocks > (long)sms * 8) blocks = (long)sms * 8;
     sumsq_kernel<<<(int)blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx, acc);
     LRQ_CUDA_TRY(cudaGetLastError());
