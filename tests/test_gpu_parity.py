@@ -276,3 +276,35 @@ def test_ars_metric_and_choice(P, orc, M, K, n_sal, thr):
     Jo, ko = orc.fluctuation_metric(bf16_bits_to_f64(xb), thr)
     assert abs(J.item() - Jo) <= 1e-6 * Jo
     assert abs(Jo - thr) > 1e-4 * thr and kind.item() == ko
+
+
+# ------------------------------------------------------------------------------- layouts and edges
+def test_qlinear_strided_input_and_output(P):
+    # X and Y as column slices of wider buffers (ldx > K, ldy > N): the TMA store path must honour ldy and must
+    # not touch the columns beside Y
+    spec = LayerSpec("s", 81, 300, 512, 264, 4, 8, 0, "hadamard", 128)
+    layer, _ = PU.gpu_layer(spec, spec.weights(), P)
+    Xc = PU.bf16_to_device(spec.activations())
+    ref = P.lrq_qlinear(layer, Xc, P.F32)
+    Xw = torch.zeros((300, 640), dtype=torch.bfloat16, device="cuda")
+    Xw[:, 64:576] = Xc
+    Yw = torch.full((300, 320), -7.0, dtype=torch.float32, device="cuda")
+    out = P.lrq_qlinear(layer, Xw[:, 64:576], P.F32, out=Yw[:, 32:296])
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref)
+    assert (Yw[:, :32] == -7.0).all() and (Yw[:, 296:] == -7.0).all()
+    assert P.lrq_device_status() == 0
+
+
+@pytest.mark.parametrize("M", [1, 127, 128, 129, 257])
+def test_qlinear_token_counts_around_a_tile(P, M):
+    # one token, and counts just below / at / above the 128-row CTA tile and the 256-row pair tile; the rows of
+    # a larger batch are independent, so each must equal the first M rows of the M = 300 result
+    spec = LayerSpec("m", 82, 300, 256, 264, 3, 4, 128, "hadamard", 256)
+    layer, _ = PU.gpu_layer(spec, spec.weights(), P)
+    X = PU.bf16_to_device(spec.activations())
+    full = P.lrq_qlinear(layer, X, P.F32)
+    part = P.lrq_qlinear(layer, X[:M].contiguous(), P.F32)
+    torch.cuda.synchronize()
+    assert torch.equal(part, full[:M])
+    assert P.lrq_device_status() == 0
