@@ -41,7 +41,7 @@ namespace {
 using namespace lrq_tc;
 
 constexpr int BM_CTA = 128;                  // token rows per CTA; the pair's tile has 256
-constexpr int BN = 256;                      // output channels per tile
+constexpr int BN = 256;                      // output channels per tile (template BN_T: 256, or 128 for small problems)
 constexpr int BN_CTA = 128;                  // weight rows decoded per CTA
 constexpr int BK = 64;
 constexpr int STAGES = 4;                    // bf16 operand stages
@@ -75,7 +75,6 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STA
                               (size_t)CSTAGES * (AC_STAGE_BYTES + WC_STAGE_BYTES) + sizeof(SharedCtl);
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
-constexpr uint32_t IDESC = umma_idesc_bf16(2 * BM_CTA, BN, false, false);
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     uint32_t d;
@@ -223,7 +222,7 @@ struct Params {
     void* Y; long ldy; int M, N, K, G, y_dtype; int* status;
 };
 
-template <int A_BITS, int W_BITS>
+template <int A_BITS, int W_BITS, int BN_T>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmY) {
@@ -239,12 +238,14 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                       // 0: issues the MMAs, 1: its peer
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int tiles_m = (p.M + 2 * BM_CTA - 1) / (2 * BM_CTA), tiles_n = (p.N + BN - 1) / BN;
+    constexpr int BN_CTA_T = BN_T / 2;                              // weight rows decoded per CTA: 128 or 64
+    constexpr uint32_t IDESC = umma_idesc_bf16(2 * BM_CTA, BN_T, false, false);
+    const int tiles_m = (p.M + 2 * BM_CTA - 1) / (2 * BM_CTA), tiles_n = (p.N + BN_T - 1) / BN_T;
     const int num_tiles = tiles_m * tiles_n;
     const int kblocks = p.K / BK;
     constexpr int NLEV = 1 << W_BITS;
     constexpr int AC_ROW_BYTES = BK * A_BITS / 8;                   // 64 or 32 code bytes per token and k-block
-    constexpr uint32_t CODE_TX_BYTES = BM_CTA * AC_ROW_BYTES + WC_STAGE_BYTES;
+    constexpr uint32_t CODE_TX_BYTES = BM_CTA * AC_ROW_BYTES + BN_CTA_T * (BK / 2);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < CSTAGES; ++s) {
@@ -279,7 +280,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
                 const int m_base = (tile % tiles_m) * 2 * BM_CTA + (int)rank * BM_CTA;
-                const int n_base = (tile / tiles_m) * BN + (int)rank * BN_CTA;
+                const int n_base = (tile / tiles_m) * BN_T + (int)rank * BN_CTA_T;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int cs = it % CSTAGES;
                     ok = mbar_wait<200>(smem_u32(&ctl->cempty[cs]), ((it / CSTAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 1);
@@ -310,7 +311,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                 ok = mbar_wait_cluster<64>(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, p.status, 4);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN_T);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
                     ok = mbar_wait_cluster<32>(smem_u32(&ctl->full[s]), (it / STAGES) & 1, &ctl->abort_flag, p.status, 5);
@@ -333,19 +334,22 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         // latencies overlap the other's arithmetic.  A group's k-blocks are every second one of the CTA's
         // running count, across tile boundaries too, so ring slots and phases advance by fixed steps.
         const int t = threadIdx.x - B_WARP0 * 32;                  // 0..255
-        const int grp = t >> 7, row = t & 127;                     // k-block parity served, row of the CTA's 128
+        // 256-wide tiles: a thread decodes a whole row of the CTA's 128 (two 32-code halves); 128-wide tiles: the
+        // CTA has 64 rows and two threads share one, a half each
+        constexpr int HALVES = BN_T == 256 ? 2 : 1;
+        const int grp = t >> 7, row = BN_T == 256 ? (t & 127) : ((t & 127) >> 1), h0 = BN_T == 256 ? 0 : (t & 1);
         const int ngrp = p.K / p.G, kb_per_grp = p.G / BK;
-        // the row's eight 16-byte chunk slots in a swizzled stage, and its 32 code bytes in a code stage
-        uint32_t off[8];
+        // the row's 16-byte chunk slots in a swizzled stage, and its code bytes in a code stage
+        uint32_t off[4 * HALVES];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) off[c] = swz(row, c);
-        const uint32_t sB0 = smem_u32(sB), sWc0 = smem_u32(sWc) + (uint32_t)row * (BK / 2);
+        for (int c = 0; c < 4 * HALVES; ++c) off[c] = swz(row, 4 * h0 + c);
+        const uint32_t sB0 = smem_u32(sB), sWc0 = smem_u32(sWc) + (uint32_t)row * (BK / 2) + (uint32_t)h0 * 16;
         RingPos ring(grp);
         uint32_t it0 = 0;
         bool ok = true, have_next = false;
         float4 raw[NLEV / 4];
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, it0 += kblocks) {
-            const int n_base = (tile / tiles_m) * BN + (int)rank * BN_CTA;
+            const int n_base = (tile / tiles_m) * BN_T + (int)rank * BN_CTA_T;
             const int n = min(n_base + row, p.N - 1);               // rows past N decode a valid table; never stored
             const float4* tab = reinterpret_cast<const float4*>(p.levels + (size_t)n * ngrp * NLEV);
             const int kb0 = (grp ^ (int)it0) & 1;
@@ -362,7 +366,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             have_next = false;
             if (ngrp == 1 && tile + num_pairs < num_tiles) {
                 // per-channel tables: the next tile's table is fetched now, a whole tile before it is needed
-                const int nn = min(((tile + num_pairs) / tiles_m) * BN + (int)rank * BN_CTA + row, p.N - 1);
+                const int nn = min(((tile + num_pairs) / tiles_m) * BN_T + (int)rank * BN_CTA_T + row, p.N - 1);
                 const float4* tn = reinterpret_cast<const float4*>(p.levels + (size_t)nn * NLEV);
 #pragma unroll
                 for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tn + j);
@@ -391,14 +395,14 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                 }
                 ok = mbar_wait_warp<64>(smem_u32(&ctl->cfull[ring.cs]), ring.cph, &ctl->abort_flag, p.status, 2);
                 if (!ok) break;
-                uint4 cw2[2];
-                lds128(sWc0 + ring.cs * WC_STAGE_BYTES, cw2[0]);
-                lds128(sWc0 + ring.cs * WC_STAGE_BYTES + 16, cw2[1]);
+                uint4 cw2[HALVES];
+#pragma unroll
+                for (int h = 0; h < HALVES; ++h) lds128(sWc0 + ring.cs * WC_STAGE_BYTES + 16 * h, cw2[h]);
                 ok = mbar_wait_warp<64>(smem_u32(&ctl->empty[ring.s]), ring.ph ^ 1, &ctl->abort_flag, p.status, 3);
                 if (!ok) break;
                 const uint32_t dst = sB0 + ring.s * B_STAGE_BYTES;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                for (int h = 0; h < HALVES; ++h) {
                     const uint4 cw = cw2[h];
                     uint32_t o[16];
                     decode_w<W_BITS, A_BITS == 4>(cw.x, L, o); decode_w<W_BITS, A_BITS == 4>(cw.y, L, o + 4);
@@ -484,11 +488,11 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         const bool has_ws = p.wscale != nullptr, has_bias = p.bias != nullptr;
         uint32_t t = 0, nstore = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++t) {
-            const int m0 = (tile % tiles_m) * 2 * BM_CTA + (int)rank * BM_CTA, n0 = (tile / tiles_m) * BN;
+            const int m0 = (tile % tiles_m) * 2 * BM_CTA + (int)rank * BM_CTA, n0 = (tile / tiles_m) * BN_T;
             const int buf = t & 1;
             // stage the tile's per-column terms (wsum, wscale, bias) in shared memory
             float (*col)[BN] = ctl->col[buf];
-            for (int c = et; c < BN; c += NUM_EPI_WARPS * 32) {
+            for (int c = et; c < BN_T; c += NUM_EPI_WARPS * 32) {
                 const int n = n0 + c;
                 const bool okc = n < p.N;
                 col[0][c] = okc ? __ldg(p.wsum + n) : 0.f;
@@ -506,10 +510,10 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
             tc_fence_after();
             if (okw) {
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+                for (int c0 = 0; c0 < BN_T; c0 += 32) {
                     if (n0 + c0 >= p.N) break;                     // warp-uniform
                     uint32_t acc[32];
-                    tc_ld32(tmem_base + ((uint32_t)(ew * 32) << 16) + (uint32_t)(buf * BN + c0), acc);
+                    tc_ld32(tmem_base + ((uint32_t)(ew * 32) << 16) + (uint32_t)(buf * BN_T + c0), acc);
                     tc_wait_ld();
                     f32x2 yq[16];
 #pragma unroll
@@ -609,9 +613,9 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
     }
 }
 
-template <int A_BITS, int W_BITS>
+template <int A_BITS, int W_BITS, int BN_T>
 lrq_status launch(const Params& p, const CUtensorMap& tmA, const CUtensorMap& tmW, const CUtensorMap& tmY, int num_tiles, cudaStream_t st) {
-    auto kern = qgemm_tc_kernel<A_BITS, W_BITS>;
+    auto kern = qgemm_tc_kernel<A_BITS, W_BITS, BN_T>;
     static int max_pairs = 0;                 // per process; the library targets identical GPUs
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -653,15 +657,29 @@ lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const
     p.status = lrq_status_word();
     // code matrices as byte tensors: a tile is 128 rows by one k-block of codes
     const uint64_t a_row = (uint64_t)L->K * ab / 8, w_row = (uint64_t)L->K / 2;
+    // Tile width.  A 128-wide tile was measured at about 0.87 of the time of a 256-wide one (the weight decode
+    // halves; the activation expansion, the hand-overs and the epilogue set-up do not), so it only pays when it
+    // cuts the number of rounds of tiles over the CTA pairs: small M with a narrow or ragged N (80 wide tiles on
+    // 74 pairs are two rounds, the same work as 144 narrow tiles is two cheaper rounds).
+    int dev = 0, sms = 0;
+    LRQ_CUDA_TRY(cudaGetDevice(&dev));
+    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const long pairs_avail = sms / 2 > 0 ? sms / 2 : 1;
+    const long tiles_m = (M + 2 * BM_CTA - 1) / (2 * BM_CTA);
+    const long t256 = tiles_m * ((L->N + 255) / 256), t128 = tiles_m * ((L->N + 127) / 128);
+    const long r256 = (t256 + pairs_avail - 1) / pairs_avail, r128 = (t128 + pairs_avail - 1) / pairs_avail;
+    const bool narrow = 0.87 * (double)r128 < (double)r256 - 1e-9;
     CUtensorMap tmA, tmW;
     if (!lrq_tma::make_map_2d(&tmA, a_codes, 1, (uint64_t)M, a_row, a_row, BK * ab / 8, BM_CTA, false)) return LRQ_ERR_CUDA;
-    if (!lrq_tma::make_map_2d(&tmW, L->codes, 1, (uint64_t)L->N, w_row, w_row, BK / 2, BN_CTA, false)) return LRQ_ERR_CUDA;
+    if (!lrq_tma::make_map_2d(&tmW, L->codes, 1, (uint64_t)L->N, w_row, w_row, BK / 2, narrow ? 64 : 128, false)) return LRQ_ERR_CUDA;
     // fp32 outputs leave through TMA stores of 32 x 32 tiles; 16-bit outputs are stored directly (the map is then unused)
     CUtensorMap tmY = tmW;
     if (dt == LRQ_F32 && !lrq_tma::make_map_2d(&tmY, Y, 4, (uint64_t)M, (uint64_t)L->N, (uint64_t)ldy, 32, 32, true)) return LRQ_ERR_CUDA;
-    const int tiles = ((M + 2 * BM_CTA - 1) / (2 * BM_CTA)) * ((L->N + BN - 1) / BN);
-    if (ab == 8 && L->w_bits == 4) return launch<8, 4>(p, tmA, tmW, tmY, tiles, st);
-    if (ab == 8) return launch<8, 3>(p, tmA, tmW, tmY, tiles, st);
-    if (ab == 4 && L->w_bits == 4) return launch<4, 4>(p, tmA, tmW, tmY, tiles, st);
-    return launch<4, 3>(p, tmA, tmW, tmY, tiles, st);
+    const int tiles = (int)(narrow ? t128 : t256);
+#define LRQ_GO(AB, WB) return narrow ? launch<AB, WB, 128>(p, tmA, tmW, tmY, tiles, st) : launch<AB, WB, 256>(p, tmA, tmW, tmY, tiles, st)
+    if (ab == 8 && L->w_bits == 4) LRQ_GO(8, 4);
+    if (ab == 8) LRQ_GO(8, 3);
+    if (ab == 4 && L->w_bits == 4) LRQ_GO(4, 4);
+    LRQ_GO(4, 3);
+#undef LRQ_GO
 }
