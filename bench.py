@@ -220,12 +220,12 @@ def run_cuda(args):
         Xs_host.append(x_cache[key][0])
         Xs.append(x_cache[key][1])
         del Wd
-    ydt = P.F32
+    ydt, y_torch = out_dtype(P, args.out_dtype)
     y_cache = {}
     for s in specs:                                   # outputs: one buffer per distinct N (reused across blocks)
         key = s.N if args.config == 4 else s.seed
         if key not in y_cache:
-            y_cache[key] = torch.empty((s.M, s.N), dtype=torch.float32, device=dev)
+            y_cache[key] = torch.empty((s.M, s.N), dtype=y_torch, device=dev)
         Ys.append(y_cache[key])
     plan = P.StackPlan(layers, Xs, Ys, ydt)
     ws = torch.empty(plan.need, dtype=torch.uint8, device=dev)
@@ -289,7 +289,7 @@ def run_cuda(args):
     uniq_y = {id(y): y for y in Ys}
     y_host = {k: torch.empty(y.shape, dtype=y.dtype).pin_memory() for k, y in uniq_y.items()}
     h2d = sum(h.numel() * 2 for h, _ in uniq_x.values())
-    d2h = sum(y.numel() * 4 for y in uniq_y.values())
+    d2h = sum(y.numel() * y.element_size() for y in uniq_y.values())
 
     def e2e_step():
         for h, d in uniq_x.values():
@@ -353,7 +353,7 @@ def run_cuda(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_name(args.config), "layers": len(specs), "out_dtype": "f32",
+            "config": {"workload": workload_name(args.config), "layers": len(specs), "out_dtype": args.out_dtype,
                        "l2": "flushed between timed steps (512 MiB fill outside the timed events)",
                        "launch": "one CUDA graph replay per step" if graph is not None else "stream-ordered launches",
                        "parallelism": f"replicated batch x{world}, no collective"},
@@ -394,14 +394,15 @@ def run_kernel(args):
     if M > X.shape[0]:
         X = X.repeat((M + X.shape[0] - 1) // X.shape[0], 1)[:M].contiguous()
     rq = P.lrq_rotate_quantize_act(X, kind, s.a_bits, s.had_block, R)
-    Y = torch.empty((M, s.N), dtype=torch.float32, device=dev)
+    ydt, y_torch = out_dtype(P, args.out_dtype)
+    Y = torch.empty((M, s.N), dtype=y_torch, device=dev)
     ws = torch.empty(max(256, L.workspace_bytes(M)), dtype=torch.uint8, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     if args.kernel == "rotq":
         fn = lambda: P.lrq_rotate_quantize_act(X, kind, s.a_bits, s.had_block, R, workspace=ws, stream=stream, out=rq)
         units, unit = M * (2.0 * s.K + s.K * s.a_bits / 8.0 + 8.0) / 1e9, "GB/s"
     elif args.kernel == "qgemm":
-        fn = lambda: P.lrq_qgemm_codes(L, rq[0], rq[1], rq[2], P.F32, args.gemm_impl, Y, stream)
+        fn = lambda: P.lrq_qgemm_codes(L, rq[0], rq[1], rq[2], ydt, args.gemm_impl, Y, stream)
         units, unit = 2.0 * M * s.N * s.K / 1e12, "TFLOP/s"
     elif args.kernel == "ars":
         fn = lambda: P.lrq_ars_select(X, 1.0, stream)
@@ -417,7 +418,7 @@ def run_kernel(args):
         if args.kernel == "rotq":
             call = lambda: P.lrq_rotate_quantize_act(X, kind, s.a_bits, s.had_block, R, workspace=ws, out=rq)
         elif args.kernel == "qgemm":
-            call = lambda: P.lrq_qgemm_codes(L, rq[0], rq[1], rq[2], P.F32, args.gemm_impl, Y)
+            call = lambda: P.lrq_qgemm_codes(L, rq[0], rq[1], rq[2], ydt, args.gemm_impl, Y)
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             call()
@@ -431,10 +432,15 @@ def run_kernel(args):
     torch.cuda.synchronize()
     ms = [a.elapsed_time(b) for a, b in ts]
     print(json.dumps({"kernel": args.kernel, "layer": s.name, "M": M, "K": s.K, "N": s.N, "rot": s.rot,
-                      "had_block": s.had_block, "w_bits": s.w_bits, "a_bits": s.a_bits,
+                      "had_block": s.had_block, "w_bits": s.w_bits, "a_bits": s.a_bits, "out_dtype": args.out_dtype,
                       "ms_mean": float(np.mean(ms)), "ms_min": float(np.min(ms)),
                       "rate_mean": units / (float(np.mean(ms)) * 1e-3), "rate_best": units / (float(np.min(ms)) * 1e-3),
                       "unit": unit, "status": P.lrq_device_status()}))
+
+
+def out_dtype(P, name):
+    import torch
+    return {"f32": (P.F32, torch.float32), "f16": (P.F16, torch.float16), "bf16": (P.BF16, torch.bfloat16)}[name]
 
 
 def main():
@@ -449,6 +455,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph replay of the step")
     ap.add_argument("--kernel", default=None, choices=["rotq", "qgemm", "tlq", "ars"], help="time one kernel only")
     ap.add_argument("--layer", type=int, default=0, help="layer index of the workload for --kernel")
+    ap.add_argument("--out-dtype", default="f32", choices=["f32", "f16", "bf16"], help="type of the layer outputs Y")
     ap.add_argument("--tokens", type=int, default=0, help="override M for --kernel")
     args = ap.parse_args()
     if args.kernel:

@@ -537,22 +537,38 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                             }
                             y[2 * j] = a0; y[2 * j + 1] = a1;
                         }
-                        const int nvalid = min(32, p.N - (n0 + c0));
-                        if (p.y_dtype == LRQ_F32 && nvalid < 32) {
-                            float* dst = static_cast<float*>(p.Y) + (size_t)m * p.ldy + n0 + c0;
+                    }
+                    // A lane holds 32 consecutive outputs of its own row; stored as they are, every store would
+                    // touch 32 different rows, a sector or less each.  The warp lays its chunk out in shared memory
+                    // (rows of 128 bytes, 128-byte swizzle: conflict-free) and one lane hands it to the TMA, which
+                    // writes whole lines, clips rows past M and columns past N, and runs while the next chunk is
+                    // prepared.  fp32: one 32 x 32 tile per chunk; 16-bit: two chunks side by side, 32 rows x 64.
+                    if (m0 + ew * 32 < p.M) {                          // warp-uniform; every store starts inside Y
+                        const uint32_t tile = smem_u32(sEpi) + (uint32_t)((ew * EPI_TILES + (nstore & 1)) * EPI_TILE_BYTES);
+                        if (p.y_dtype == LRQ_F32) {
+                            if (lane == 0) tma_store_wait_read<EPI_TILES - 1>();     // the store that last read this tile is done with it
+                            __syncwarp();
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                float a, b; unpack2(y[j], a, b);
-                                if (2 * j < nvalid) dst[2 * j] = a;
-                                if (2 * j + 1 < nvalid) dst[2 * j + 1] = b;
+                            for (int j = 0; j < 8; ++j) {
+                                float a, b, c2, d;
+                                unpack2(yq[2 * j], a, b); unpack2(yq[2 * j + 1], c2, d);
+                                sts128(tile + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4)), __float_as_uint(a), __float_as_uint(b),
+                                       __float_as_uint(c2), __float_as_uint(d));
                             }
-                        } else if (p.y_dtype == LRQ_F32) {
-                            // handled below by the whole warp (rows past M take part in the exchange, not in the stores)
+                            fence_async_smem();
+                            __syncwarp();
+                            if (lane == 0) tma_store_2d(&tmY, n0 + c0, m0 + ew * 32, tile);
+                            ++nstore;
                         } else {
+                            const int half = (c0 >> 5) & 1;
+                            if (half == 0) {
+                                if (lane == 0) tma_store_wait_read<EPI_TILES - 1>();
+                                __syncwarp();
+                            }
                             uint32_t h[16];
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
-                                float a, b; unpack2(y[j], a, b);
+                                float a, b; unpack2(yq[j], a, b);
                                 if (p.y_dtype == LRQ_BF16) {
                                     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
                                     h[j] = *reinterpret_cast<uint32_t*>(&v);
@@ -561,36 +577,17 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                                     h[j] = *reinterpret_cast<uint32_t*>(&v);
                                 }
                             }
-                            uint16_t* dst = static_cast<uint16_t*>(p.Y) + (size_t)m * p.ldy + n0 + c0;
-                            if (nvalid == 32) {
 #pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    reinterpret_cast<uint4*>(dst)[j] = make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = (uint16_t)(h[j >> 1] >> (16 * (j & 1)));
+                            for (int j = 0; j < 4; ++j)
+                                sts128(tile + (uint32_t)(lane * 128 + (((half * 4 + j) ^ (lane & 7)) << 4)), h[4 * j], h[4 * j + 1],
+                                       h[4 * j + 2], h[4 * j + 3]);
+                            if (half == 1 || n0 + c0 + 32 >= p.N) {    // the pair is complete, or its second chunk lies past N
+                                fence_async_smem();
+                                __syncwarp();
+                                if (lane == 0) tma_store_2d(&tmY, n0 + (c0 & ~63), m0 + ew * 32, tile);
+                                ++nstore;
                             }
                         }
-                    }
-                    if (p.y_dtype == LRQ_F32 && n0 + c0 + 32 <= p.N && m0 + ew * 32 < p.M) {     // warp-uniform; every store starts inside Y
-                        // A lane holds 32 consecutive outputs of its own row; stored as they are, every store would
-                        // touch 32 different rows, half a sector each.  The warp lays its 32 x 32 chunk out in shared
-                        // memory (rows of 128 bytes, 128-byte swizzle: conflict-free) and one lane hands it to the TMA,
-                        // which writes whole lines, clips rows past M, and runs while the next chunk is prepared.
-                        const uint32_t tile = smem_u32(sEpi) + (uint32_t)((ew * EPI_TILES + (nstore & 1)) * EPI_TILE_BYTES);
-                        if (lane == 0) tma_store_wait_read<EPI_TILES - 1>();     // the store that last read this tile is done with it
-                        __syncwarp();
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            float a, b, c2, d;
-                            unpack2(yq[2 * j], a, b); unpack2(yq[2 * j + 1], c2, d);
-                            sts128(tile + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4)), __float_as_uint(a), __float_as_uint(b),
-                                   __float_as_uint(c2), __float_as_uint(d));
-                        }
-                        fence_async_smem();
-                        __syncwarp();
-                        if (lane == 0) tma_store_2d(&tmY, n0 + c0, m0 + ew * 32, tile);
-                        ++nstore;
                     }
                 }
             }
@@ -672,9 +669,9 @@ lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const
     CUtensorMap tmA, tmW;
     if (!lrq_tma::make_map_2d(&tmA, a_codes, 1, (uint64_t)M, a_row, a_row, BK * ab / 8, BM_CTA, false)) return LRQ_ERR_CUDA;
     if (!lrq_tma::make_map_2d(&tmW, L->codes, 1, (uint64_t)L->N, w_row, w_row, BK / 2, narrow ? 64 : 128, false)) return LRQ_ERR_CUDA;
-    // fp32 outputs leave through TMA stores of 32 x 32 tiles; 16-bit outputs are stored directly (the map is then unused)
-    CUtensorMap tmY = tmW;
-    if (dt == LRQ_F32 && !lrq_tma::make_map_2d(&tmY, Y, 4, (uint64_t)M, (uint64_t)L->N, (uint64_t)ldy, 32, 32, true)) return LRQ_ERR_CUDA;
+    // outputs leave through TMA stores of 32-row tiles, 128 bytes wide (32 fp32 or 64 16-bit columns)
+    CUtensorMap tmY;
+    if (!lrq_tma::make_map_2d(&tmY, Y, (int)es, (uint64_t)M, (uint64_t)L->N, (uint64_t)ldy, dt == LRQ_F32 ? 32 : 64, 32, true)) return LRQ_ERR_CUDA;
     const int tiles = (int)(narrow ? t128 : t256);
 #define LRQ_GO(AB, WB) return narrow ? launch<AB, WB, 128>(p, tmA, tmW, tmY, tiles, st) : launch<AB, WB, 256>(p, tmA, tmW, tmY, tiles, st)
     if (ab == 8 && L->w_bits == 4) LRQ_GO(8, 4);

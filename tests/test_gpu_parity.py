@@ -279,17 +279,20 @@ def test_ars_metric_and_choice(P, orc, M, K, n_sal, thr):
 
 
 # ------------------------------------------------------------------------------- layouts and edges
-def test_qlinear_strided_input_and_output(P):
-    # X and Y as column slices of wider buffers (ldx > K, ldy > N): the TMA store path must honour ldy and must
-    # not touch the columns beside Y
+@pytest.mark.parametrize("dt", ["F32", "F16", "BF16"])
+def test_qlinear_strided_input_and_output(P, dt):
+    # X and Y as column slices of wider buffers (ldx > K, ldy > N; N = 264 ends inside a 32- and a 64-column store
+    # tile): the TMA store path must honour ldy and must not touch the columns beside Y
+    code = getattr(P, dt)
+    tdt = {"F32": torch.float32, "F16": torch.float16, "BF16": torch.bfloat16}[dt]
     spec = LayerSpec("s", 81, 300, 512, 264, 4, 8, 0, "hadamard", 128)
     layer, _ = PU.gpu_layer(spec, spec.weights(), P)
     Xc = PU.bf16_to_device(spec.activations())
-    ref = P.lrq_qlinear(layer, Xc, P.F32)
+    ref = P.lrq_qlinear(layer, Xc, code)
     Xw = torch.zeros((300, 640), dtype=torch.bfloat16, device="cuda")
     Xw[:, 64:576] = Xc
-    Yw = torch.full((300, 320), -7.0, dtype=torch.float32, device="cuda")
-    out = P.lrq_qlinear(layer, Xw[:, 64:576], P.F32, out=Yw[:, 32:296])
+    Yw = torch.full((300, 320), -7.0, dtype=tdt, device="cuda")
+    out = P.lrq_qlinear(layer, Xw[:, 64:576], code, out=Yw[:, 32:296])
     torch.cuda.synchronize()
     assert torch.equal(out, ref)
     assert (Yw[:, :32] == -7.0).all() and (Yw[:, 296:] == -7.0).all()
