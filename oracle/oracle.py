@@ -21,7 +21,7 @@ _LIB = os.path.join(_HERE, "liblrq_oracle.so")
 __all__ = [
     "build", "num_threads", "hadamard_matrix", "rotate_hadamard_explicit", "rotate_hadamard_fwht",
     "rotate_dense", "quantize_act", "dequantize_act", "level_value", "tlq_quantize", "qmatmul",
-    "TLQResult", "qlinear", "smooth", "fluctuation_metric",
+    "TLQResult", "qlinear", "smooth", "fluctuation_metric", "rotate_weights",
 ]
 
 
@@ -108,6 +108,22 @@ def smooth(X, p):
     Y = np.empty_like(X)
     _L().orc_smooth(xp, M, K, pp, Y.ctypes.data_as(_dp))
     return Y
+
+
+def rotate_weights(W, colmul=None, rot: str = "hadamard", had_block: int = 0, R=None):
+    """The weight side of Eq. 2, (X R)(W R)^T = X W^T: the rows of W diag(colmul) mapped by the layer's rotation
+    (Sec. 3.2; colmul is the reciprocal of the activations' smoothing multipliers, Sec. 5.1).  The same maps the
+    activations take, applied to weight rows."""
+    W = np.asarray(W, dtype=np.float64)
+    if colmul is not None:
+        W = smooth(W, np.asarray(colmul, dtype=np.float64))
+    if rot == "hadamard":
+        return rotate_hadamard_fwht(W, had_block)
+    if rot == "dense":
+        return rotate_dense(W, R)
+    if rot == "none":
+        return W.copy()
+    raise ValueError(rot)
 
 
 def fluctuation_metric(X, thr: float = 1.0):

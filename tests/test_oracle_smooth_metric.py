@@ -3,7 +3,7 @@ fluctuation metric J with its threshold rule (Sec. 4.2, Eqs. 11-12)."""
 import numpy as np
 import pytest
 
-from lrq_workloads import make_activations, make_weights, bf16_bits_to_f64
+from lrq_workloads import make_activations, make_orthogonal, make_weights, bf16_bits_to_f64
 
 
 def test_smoothing_leaves_the_product_unchanged(orc):
@@ -20,6 +20,32 @@ def test_smoothing_leaves_the_product_unchanged(orc):
     Yr = orc.rotate_hadamard_fwht(Xs, 128) @ orc.rotate_hadamard_fwht(Ws, 128).T
     assert np.allclose(Yr, ref, rtol=1e-11, atol=1e-11 * np.abs(ref).max())
     assert np.array_equal(orc.smooth(X, np.ones(256)), X)     # unit multipliers change nothing
+
+
+@pytest.mark.parametrize("rot,B", [("hadamard", 64), ("hadamard", 256), ("dense", 0), ("none", 0)])
+def test_rotated_weights_keep_the_layer_product(orc, rot, B):
+    # Eq. 2 with the smoothing of Sec. 5.1: (X diag(p) R)(W diag(1/p) R)^T = X W^T for an orthogonal R.  A dropped
+    # multiplier, a transposed R or a missing 1/sqrt(B) on either side breaks the identity.
+    rng = np.random.default_rng(5)
+    K = 256
+    X = bf16_bits_to_f64(make_activations(11, 6, K))
+    W = make_weights(12, 10, K).astype(np.float64)
+    p = rng.uniform(0.2, 4.0, K)
+    R = make_orthogonal(13, K) if rot == "dense" else None
+    Wr = orc.rotate_weights(W, 1.0 / p, rot, B, R)
+    Xs = orc.smooth(X, p)
+    Xr = {"hadamard": lambda: orc.rotate_hadamard_fwht(Xs, B), "dense": lambda: orc.rotate_dense(Xs, R),
+          "none": lambda: Xs}[rot]()
+    ref = X @ W.T
+    assert np.allclose(Xr @ Wr.T, ref, rtol=1e-11, atol=1e-11 * np.abs(ref).max())
+    # against the explicit matrices (library product), and the norm of every row is kept by the rotation
+    if rot == "hadamard":
+        Hb = np.kron(np.eye(K // B), orc.hadamard_matrix(B))
+        assert np.allclose(Wr, (W / p) @ Hb, rtol=1e-12, atol=1e-15)
+    if rot == "dense":
+        assert np.allclose(Wr, (W / p) @ R, rtol=1e-12, atol=1e-15)
+    assert np.allclose(np.linalg.norm(Wr, axis=1), np.linalg.norm(W / p, axis=1), rtol=1e-12)
+    assert np.array_equal(orc.rotate_weights(W, None, "none"), W)
 
 
 def test_smoothing_tames_salient_channels(orc):
