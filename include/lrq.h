@@ -130,6 +130,23 @@ lrq_status lrq_ars_select(const void* X_bf16, int M, int K, long ldx, double thr
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Weight side of the rotation identity (Sec. 3.2, Eq. 2: (X R)(W R)^T = X W^T), offline:
+ *   W_rot = W diag(colmul) R,   evaluated in fp64 and rounded once to fp32,
+ * the matrix lrq_tlq_quantize_weights reads.  R is the layer's rotation: blockdiag(H_B) (Eq. 3), the
+ * stored bf16 matrix of the dense case (the same array lrq_act_params.R_bf16 points to, so both
+ * sides of Eq. 2 use one R), or the identity.  colmul absorbs the smoothing of Sec. 5.1: with
+ * activations multiplied by prescale[k], pass colmul[k] = 1 / prescale[k].
+ *   W       dev float [N,ldw], ldw >= K
+ *   colmul  dev float [K], nullable (all ones)
+ *   R_bf16  dev bf16 [K,K] row-major, LRQ_ROT_DENSE only
+ *   W_rot   dev float [N,ldo], ldo >= K (out); may be W itself except for LRQ_ROT_DENSE
+ * LRQ_ROT_HADAMARD: had_block a power of two dividing K, K <= 25600 (the row is held in shared
+ * memory as fp64).  No workspace.
+ * ------------------------------------------------------------------------------------------- */
+lrq_status lrq_rotate_weights(const float* W, int N, int K, long ldw, const float* colmul, lrq_rot_kind kind,
+                              int had_block, const void* R_bf16, float* W_rot, long ldo, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * lrq_rotate_quantize_act for callers that cannot hand over device scratch.
  *
  * (The paper has no counterpart; this entry point exists for integration reasons only.)

@@ -21,6 +21,7 @@ EXPORTS = [
     "lrq_tlq_quantize_weights", "lrq_act_workspace_bytes", "lrq_rotate_quantize_act", "lrq_layer_create",
     "lrq_layer_destroy", "lrq_workspace_bytes", "lrq_qlinear", "lrq_qlinear_stack", "lrq_qgemm_codes",
     "lrq_device_status", "lrq_status_string", "lrq_version", "lrq_rotate_quantize_act_static", "lrq_ars_select",
+    "lrq_rotate_weights",
 ]
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -72,6 +73,7 @@ def load_library() -> C.CDLL:
                                       C.POINTER(vp), ci, C.POINTER(cl), vp, sz, vp]
     lib.lrq_qgemm_codes.argtypes = [vp, vp, vp, vp, ci, vp, ci, cl, ci, vp]
     lib.lrq_ars_select.argtypes = [vp, ci, ci, cl, C.c_double, vp, vp, vp, sz, vp]
+    lib.lrq_rotate_weights.argtypes = [vp, ci, ci, cl, vp, ci, ci, vp, vp, cl, vp]
     lib.lrq_device_status.argtypes = [vp]
     lib.lrq_status_string.argtypes = [ci]
     lib.lrq_status_string.restype = C.c_char_p
@@ -150,6 +152,24 @@ def _act_params(kind: int, had_block: int, R: Optional[torch.Tensor], a_bits: in
         assert prescale.dtype == torch.float32 and prescale.is_contiguous()
     return _ActParams(int(kind), int(had_block), 0 if R is None else R.data_ptr(), int(a_bits), int(mode),
                       0 if prescale is None else prescale.data_ptr())
+
+
+def lrq_rotate_weights(W: torch.Tensor, kind: int, had_block: int = 0, R: Optional[torch.Tensor] = None,
+                       colmul: Optional[torch.Tensor] = None, stream=None, out: Optional[torch.Tensor] = None):
+    """W diag(colmul) R in fp64, rounded to fp32: the weight side of Eq. 2 (offline).  Returns W_rot float32 [N,K]."""
+    _need_cuda(W)
+    assert W.dtype == torch.float32 and W.dim() == 2 and W.stride(1) == 1
+    N, K = W.shape
+    if R is not None:
+        assert R.dtype == torch.bfloat16 and R.shape == (K, K) and R.is_contiguous()
+    if colmul is not None:
+        assert colmul.dtype == torch.float32 and colmul.shape == (K,) and colmul.is_contiguous()
+    if out is None:
+        out = torch.empty((N, K), dtype=torch.float32, device=W.device)
+    assert out.dtype == torch.float32 and out.shape == (N, K) and out.stride(1) == 1
+    _check(load_library().lrq_rotate_weights(_ptr(W), N, K, W.stride(0), _ptr(colmul), kind, had_block, _ptr(R), _ptr(out),
+                                             out.stride(0), _stream(stream)), "lrq_rotate_weights")
+    return out
 
 
 def lrq_ars_select(X: torch.Tensor, threshold: float = 1.0, stream=None):

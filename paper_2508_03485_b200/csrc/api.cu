@@ -119,6 +119,20 @@ extern "C" lrq_status lrq_ars_select(const void* X, int M, int K, long ldx, doub
                                  (cudaStream_t)cuda_stream);
 }
 
+extern "C" lrq_status lrq_rotate_weights(const float* W, int N, int K, long ldw, const float* colmul, lrq_rot_kind kind,
+                                         int had_block, const void* R_bf16, float* W_rot, long ldo, void* cuda_stream) {
+    if (!W || !W_rot || N <= 0 || K <= 0 || ldw < K || ldo < K) return LRQ_ERR_INVALID_ARG;
+    if (kind == LRQ_ROT_HADAMARD) {
+        if (had_block < 1 || (had_block & (had_block - 1)) || K % had_block) return LRQ_ERR_INVALID_ARG;
+    } else if (kind == LRQ_ROT_DENSE) {
+        if (!R_bf16) return LRQ_ERR_INVALID_ARG;
+        if (W_rot == W) return LRQ_ERR_INVALID_ARG;               // the product reads whole rows of W per output tile
+    } else if (kind != LRQ_ROT_NONE) {
+        return LRQ_ERR_INVALID_ARG;
+    }
+    return lrq_launch_rotate_weights(W, N, K, ldw, colmul, (int)kind, had_block, R_bf16, W_rot, ldo, (cudaStream_t)cuda_stream);
+}
+
 extern "C" lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size,
                                        const uint8_t* codes, const float* levels, const float* wsum,
                                        const float* wscale, const float* bias, const lrq_act_params* act) {

@@ -47,6 +47,10 @@ lrq_status lrq_launch_quantize_f32_ext(const float* Y, int M, int K, int a_bits,
 lrq_status lrq_launch_ars_metric(const void* X, int M, int K, long ldx, double thr, float* J, int* kind, double* acc,
                                  cudaStream_t st);
 
+// wrot.cu : W diag(colmul) R in fp64, rounded to fp32 (Eq. 2, weight side)
+lrq_status lrq_launch_rotate_weights(const float* W, int N, int K, long ldw, const float* colmul, int kind,
+                                     int had_block, const void* R, float* out, long ldo, cudaStream_t st);
+
 #ifdef __CUDACC__
 // Order-preserving map between fp32 and int32 (and back), so that integer min/max reductions serve floats.
 __device__ __forceinline__ int lrq_ordered_int(float f) { const int i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }

@@ -311,3 +311,54 @@ def test_qlinear_token_counts_around_a_tile(P, M):
     torch.cuda.synchronize()
     assert torch.equal(part, full[:M])
     assert P.lrq_device_status() == 0
+
+
+@pytest.mark.parametrize("N,K,rot,B,smooth", [(37, 1152, "hadamard", 128, True), (5, 12288, "hadamard", 4096, False),
+                                              (70, 384, "dense", 0, True), (130, 200, "dense", 0, False),
+                                              (9, 72, "none", 0, True), (16, 1536, "hadamard", 512, True)])
+def test_rotate_weights(P, orc, N, K, rot, B, smooth):
+    # W diag(colmul) R (Eq. 2, weight side; Sec. 5.1) against the oracle.  Both evaluate in fp64 and differ only in
+    # summation order (1e-13 relative); after the one rounding to fp32 that shows as at most one ulp, and only
+    # where the fp64 value sits next to a rounding boundary.
+    rng = np.random.default_rng(N + K)
+    W = make_weights(31, N, K)
+    c = rng.uniform(0.3, 3.0, K).astype(np.float32) if smooth else None
+    R = Rb = None
+    if rot == "dense":
+        Rb = f32_to_bf16_bits(make_orthogonal(7, K).astype(np.float32))
+        R = PU.bf16_to_device(Rb)
+    kind = {"hadamard": P.ROT_HADAMARD, "dense": P.ROT_DENSE, "none": P.ROT_NONE}[rot]
+    out = P.lrq_rotate_weights(torch.from_numpy(W).cuda(), kind, B, R, None if c is None else torch.from_numpy(c).cuda())
+    ref = orc.rotate_weights(W.astype(np.float64), None if c is None else c.astype(np.float64), rot, B,
+                             None if Rb is None else bf16_bits_to_f64(Rb))
+    got = out.cpu().numpy()
+    ref32 = ref.astype(np.float32)
+    ulp = np.spacing(np.abs(ref32)).astype(np.float64)
+    assert (np.abs(got.astype(np.float64) - ref) <= 0.5 * ulp + 1e-12 * np.abs(ref).max()).all()
+    assert (got != ref32).mean() < 1e-3
+    if rot == "hadamard":          # in place is allowed for this kind
+        Wd = torch.from_numpy(W).cuda()
+        P.lrq_rotate_weights(Wd, kind, B, None, None if c is None else torch.from_numpy(c).cuda(), out=Wd)
+        assert torch.equal(Wd, out)
+
+
+def test_rotated_and_smoothed_layer_reproduces_the_plain_product(P):
+    # End to end on the GPU: weights rotated by lrq_rotate_weights with colmul = 1/p, activations smoothed by p and
+    # rotated inside lrq_qlinear.  With 8-bit activations and 4-bit TLQ the result is a quantized estimate of X W^T;
+    # its error must be that of the quantizers (a few per cent of the output scale), far from what a mismatch of
+    # the two sides of Eq. 2 would give (order one).
+    rng = np.random.default_rng(3)
+    M, K, N, B = 200, 1152, 264, 128
+    W = make_weights(51, N, K)
+    xb = make_activations(52, M, K)
+    X = bf16_bits_to_f64(xb)
+    p = (1.0 / np.sqrt(np.abs(X).max(axis=0) + 1e-3)).astype(np.float32)
+    Wr = P.lrq_rotate_weights(torch.from_numpy(W).cuda(), P.ROT_HADAMARD, B, None, torch.from_numpy(1.0 / p).cuda())
+    grid = default_clip_grid()
+    tl = P.lrq_tlq_quantize_weights(Wr, 4, 0, 7, grid, grid)
+    layer = P.QLayer(tl, N, K, P.ROT_HADAMARD, 8, B, prescale=torch.from_numpy(p).cuda())
+    Y = P.lrq_qlinear(layer, PU.bf16_to_device(xb), P.F32).cpu().numpy().astype(np.float64)
+    ref = X @ W.astype(np.float64).T
+    err = np.linalg.norm(Y - ref) / np.linalg.norm(ref)
+    assert err < 0.2, err       # the oracle gives 0.117 on these inputs; without colmul it is 0.92
+    assert P.lrq_device_status() == 0
