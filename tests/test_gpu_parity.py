@@ -362,3 +362,40 @@ def test_rotated_and_smoothed_layer_reproduces_the_plain_product(P):
     err = np.linalg.norm(Y - ref) / np.linalg.norm(ref)
     assert err < 0.2, err       # the oracle gives 0.117 on these inputs; without colmul it is 0.92
     assert P.lrq_device_status() == 0
+
+
+def _sweep_shapes():
+    rng = np.random.default_rng(2024)
+    out = []
+    for i in range(28):
+        K = 64 * int(rng.integers(1, 25))
+        G = 128 if (K % 128 == 0 and rng.random() < 0.5) else 0
+        M = int(rng.integers(1, 900))
+        N = 8 * int(rng.integers(1, 180))
+        w_bits, a_bits = int(rng.choice([3, 4])), int(rng.choice([4, 8]))
+        dt = ["F32", "F16", "BF16"][i % 3]
+        out.append((M, K, N, w_bits, a_bits, G, dt))
+    return out
+
+
+@pytest.mark.parametrize("M,K,N,w_bits,a_bits,G,dt", _sweep_shapes())
+def test_qgemm_shape_sweep_against_cuda_core(P, M, K, N, w_bits, a_bits, G, dt):
+    # Seeded random shapes (ragged M and N, one to 24 k-blocks, both tile widths, every output type): the tcgen05
+    # kernel against the plain CUDA-core kernel on the same codes.  fp32: summation order only; 16-bit outputs:
+    # one more rounding of a value that may differ in its last fp32 bits (one 16-bit ulp).
+    B = 1
+    while K % (2 * B) == 0 and B < 128:
+        B *= 2
+    spec = LayerSpec("w", 900 + M, M, K, N, w_bits, a_bits, G, "hadamard", B)
+    layer, _ = PU.gpu_layer(spec, spec.weights(), P)
+    X = PU.bf16_to_device(spec.activations())
+    q, s, z = P.lrq_rotate_quantize_act(X, P.ROT_HADAMARD, a_bits, B)
+    code = getattr(P, dt)
+    ref = P.lrq_qgemm_codes(layer, q, s, z, code, 1).float()
+    Y = P.lrq_qgemm_codes(layer, q, s, z, code, 0).float()
+    torch.cuda.synchronize()
+    assert P.lrq_device_status() == 0
+    rms = ref.pow(2).mean().sqrt().item()
+    tol = 2e-3 * rms if dt == "F32" else (2e-3 * rms + ref.abs() * (2.0 ** -7 if dt == "BF16" else 2.0 ** -10))
+    assert ((Y - ref).abs() <= tol).all()
+    layer.close()
