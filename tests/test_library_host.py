@@ -60,7 +60,17 @@ def test_argument_checks_run_before_any_launch(lib):
     assert lib.lrq_workspace_bytes(h, 10) == 768 + 256 + 256
     assert lib.lrq_qlinear(h, fake, 10, 64, fake, 0, 8, None, 0, None) == 3       # workspace missing
     assert lib.lrq_qlinear(h, fake, 10, 64, fake, 0, 4, fake, 1 << 20, None) == 1  # ldy < N
+    assert lib.lrq_qlinear(h, fake, 0, 64, fake, 0, 64, fake, 1 << 20, None) == 1  # no tokens: an argument error, nothing launched
     lib.lrq_layer_destroy(h)
+    assert lib.lrq_rotate_quantize_act(fake, 0, 128, 128, C.byref(p), fake, fake, fake, None, 0, None) == 1
+    # weight rotation: block size must be a power of two dividing K; a dense rotation needs R and cannot run in place
+    assert lib.lrq_rotate_weights(fake, 8, 192, 192, None, 1, 128, None, fake, 192, None) == 1
+    assert lib.lrq_rotate_weights(fake, 8, 128, 128, None, 2, 0, None, fake, 128, None) == 1
+    assert lib.lrq_rotate_weights(fake, 8, 128, 128, None, 2, 0, fake, fake, 128, None) == 1
+    assert lib.lrq_rotate_weights(fake, 8, 128, 64, None, 0, 0, None, fake, 128, None) == 1      # ldw < K
+    # rotation choice: 8 bytes of workspace, K a multiple of 16
+    assert lib.lrq_ars_select(fake, 4, 128, 128, 1.0, fake, fake, None, 0, None) == 3
+    assert lib.lrq_ars_select(fake, 4, 120, 120, 1.0, fake, fake, fake, 8, None) == 2
 
 
 def test_calling_without_a_gpu_fails_loudly():
