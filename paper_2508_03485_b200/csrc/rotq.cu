@@ -416,6 +416,197 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
 }
 
 // ------------------------------------------------------------------------------------------------
+// Large blocks (B = 1024, 2048, 4096).  With five or more index bits above a thread's own 32 elements,
+// butterflies between lanes move every value through the shuffle network once per stage (20 bytes per element
+// for bits 5-9, 8 more per shared-memory stage above).  This kernel instead re-distributes the data twice
+// through shared memory and keeps every butterfly between a thread's own registers:
+//   A  a warp transposes its 32 x 32 elements (index = 32 * row + col: each thread writes its row, reads its
+//      column), after which index bits 5-9 are register butterflies;
+//   B  the U = B/1024 warps of a transform block write their columns back and every thread reads four runs of
+//      eight consecutive elements, one run per value of the block's top two index bits: bits 10-11 become
+//      register butterflies too, and the runs are what the packer needs (4 or 8 code bytes each).
+// Shared-memory traffic is 16 bytes per element in all.  Layouts: A is 32 rows of 128 bytes whose 16-byte
+// chunks are swizzled by the row (rows written with 128-bit stores, columns read word by word, both
+// conflict-free); B stores element y of the block at (y / 8) * 4 + y % 4 of one of two half-buffers chosen by
+// bit 2 of y, the second half shifted by 16 banks, so that the word-wise writes and the 128-bit reads are
+// conflict-free as well.  A warp's rows and its B words occupy the same two 2 KB pieces, so only the B reads
+// cross warps: one barrier before them; the barrier of the extremes separates them from the next group.
+// ------------------------------------------------------------------------------------------------
+template <int LOG2B, int A_BITS, int MAX_THREADS, int MIN_CTAS, bool WIDE>
+__global__ void __launch_bounds__(MAX_THREADS, MIN_CTAS)
+rotq_big_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, int mode, int tok_per_cta, int num_groups,
+                const float* __restrict__ prescale,
+                uint8_t* __restrict__ codes, float* __restrict__ scale, int32_t* __restrict__ zp) {
+    static_assert(LOG2B >= 10 && LOG2B <= 12, "block sizes 1024..4096");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    constexpr int NP = EPT / 2;
+    constexpr int U = 1 << (LOG2B - 10);             // warps per transform block
+    constexpr int HALF_OFF = U * 512 + 16;           // floats from the first half-buffer to the second
+    constexpr int UNIT_FLOATS = U * 1024 + 32;
+    const int tpt = K / EPT;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tl = tid / tpt, j = tid - tl * tpt;
+    int* ext = reinterpret_cast<int*>(smem_raw);
+    float* buf = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(ext + 3 * 2 * tok_per_cta) + 127) & ~uintptr_t(127));
+    const int wu = warp % U;                         // warp within the transform block
+    // shared-memory byte addresses: the block's buffer, this warp's two 2 KB pieces (second = first + HALF_OFF floats)
+    const uint32_t ub = (uint32_t)__cvta_generic_to_shared(buf + (warp / U) * UNIT_FLOATS);
+    const uint32_t piece0 = ub + wu * 2048;
+    // A: own row (written; chunk c at slot c ^ (lane & 7)), own column (read; word lane ^ 4 * (row & 7) of a row)
+    const uint32_t rowa = piece0 + (lane < 16 ? lane * 128 : HALF_OFF * 4 + (lane - 16) * 128);
+    const uint32_t l7s = (lane & 7) << 4;
+    const uint32_t cola = piece0 + lane * 4;
+    // B: own words (written), own runs (read)
+    const uint32_t wra = piece0 + (((lane >> 2) & 1) ? HALF_OFF * 4 : 0) + ((lane >> 3) * 4 + (lane & 3)) * 4;
+    const int tau = wu * 32 + lane;                  // thread within the block
+    const uint32_t rda = ub + tau * 16;
+    const int unit_in_token = j / (U * 32);
+
+    const unsigned seg_mask = __match_any_sync(0xffffffffu, tl);
+    const int seg_lane = __ffs(seg_mask) - 1;
+    const bool seg_leader = lane == seg_lane;
+    for (int i = tid; i < 3 * 2 * tok_per_cta; i += blockDim.x) ext[i] = (i & 1) ? INT_MIN : INT_MAX;
+    __syncthreads();
+
+    uint4 raw[4];
+    {
+        const int m = blockIdx.x * tok_per_cta + tl;
+        if (m < M) {
+            load_raw<WIDE>(X + (size_t)m * ldx + (size_t)j * EPT, raw);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) raw[i] = make_uint4(0, 0, 0, 0);
+        }
+    }
+    int it = 0;
+    for (int g = blockIdx.x; g < num_groups; g += gridDim.x, ++it) {
+        const int m = g * tok_per_cta + tl;
+        const bool live = m < M;
+        f32x2 P[NP];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                P[4 * i + c] = pack2(__uint_as_float(w[c] << 16), __uint_as_float(w[c] & 0xffff0000u));
+        }
+        if (prescale) {
+            const float4* ps = reinterpret_cast<const float4*>(prescale + (size_t)j * EPT);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 f = __ldg(ps + i);
+                P[2 * i] = mul2(P[2 * i], pack2(f.x, f.y)); P[2 * i + 1] = mul2(P[2 * i + 1], pack2(f.z, f.w));
+            }
+        }
+        {
+            const int mn = (g + (int)gridDim.x) * tok_per_cta + tl;
+            if (g + (int)gridDim.x < num_groups && mn < M) {
+                load_raw<WIDE>(X + (size_t)mn * ldx + (size_t)j * EPT, raw);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) raw[i] = make_uint4(0, 0, 0, 0);
+            }
+        }
+        // index bits 0..4 and, after the transposition, 5..9: the same register butterflies twice
+#pragma unroll
+        for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { float a, b; unpack2(P[i], a, b); P[i] = pack2(a + b, a - b); }
+#pragma unroll
+            for (int h = 1; h < NP; h <<= 1)
+#pragma unroll
+                for (int i = 0; i < NP; ++i)
+                    if (!(i & h)) { const f32x2 a = P[i], b = P[i | h]; P[i] = add2(a, b); P[i | h] = sub2(a, b); }
+            if (pass == 0) {
+                // A: rows out (chunk c of row `lane` at slot c ^ (lane & 7)), columns in
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    asm volatile("st.shared.v2.b64 [%0], {%1, %2};" :: "r"(rowa + (l7s ^ (c << 4))), "l"(P[2 * c]), "l"(P[2 * c + 1]) : "memory");
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < NP; ++i) {
+                    // rows 2i and 2i+1 of the warp's 32 x 32 elements, word `lane` of each (swizzled by the row)
+                    const int r = 2 * i;
+                    const uint32_t rb = (r < 16 ? r * 128 : HALF_OFF * 4 + (r - 16) * 128);
+                    float a, b;
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(a) : "r"((cola ^ ((r & 7) << 4)) + rb) : "memory");
+                    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(b) : "r"((cola ^ (((r + 1) & 7) << 4)) + rb + 128) : "memory");
+                    P[i] = pack2(a, b);
+                }
+                __syncwarp();                         // every lane has read its column before the words below land
+            }
+        }
+        // B: the thread's column (element 32 * i + lane of the warp's 1024) out word by word, four runs of eight in
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            float a, b;
+            unpack2(P[i], a, b);
+            asm volatile("st.shared.f32 [%0], %1;" :: "r"(wra + (2 * i) * 64), "f"(a) : "memory");
+            asm volatile("st.shared.f32 [%0], %1;" :: "r"(wra + (2 * i + 1) * 64), "f"(b) : "memory");
+        }
+        // the block's U warps meet on their own named barrier (ids 1..: barrier 0 is the CTA's)
+        if (U == 1) __syncwarp(); else asm volatile("bar.sync %0, %1;" :: "r"(1 + warp / U), "n"(U * 32) : "memory");
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(P[4 * r]), "=l"(P[4 * r + 1]) : "r"(rda + r * (U * 512)) : "memory");
+            asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(P[4 * r + 2]), "=l"(P[4 * r + 3]) : "r"(rda + r * (U * 512) + HALF_OFF * 4) : "memory");
+        }
+        // index bits 10..11: between the runs
+#pragma unroll
+        for (int h = (LOG2B == 12 ? 4 : 8); h < NP && LOG2B > 10; h <<= 1)
+#pragma unroll
+            for (int i = 0; i < NP; ++i)
+                if (!(i & h)) { const f32x2 a = P[i], b = P[i | h]; P[i] = add2(a, b); P[i | h] = sub2(a, b); }
+
+        float mn, mx;
+        unpack2(P[0], mn, mx);
+        { const float t0 = fminf(mn, mx); mx = fmaxf(mn, mx); mn = t0; }
+#pragma unroll
+        for (int i = 1; i < NP; ++i) { float x, y; unpack2(P[i], x, y); mn = min3(mn, x, y); mx = max3(mx, x, y); }
+        int* slot = ext + (it % 3) * 2 * tok_per_cta + 2 * tl;
+        {
+            const int imn = __reduce_min_sync(seg_mask, lrq_ordered_int(mn)), imx = __reduce_max_sync(seg_mask, lrq_ordered_int(mx));
+            if (seg_leader) { atomicMin(slot, imn); atomicMax(slot + 1, imx); }
+        }
+        __syncthreads();
+        TokenQ t;
+        {
+            float sc = 0.f; int z = 0;
+            t.inv = 0.f; t.negz = 0.f;
+            if (seg_leader) {
+                const float a = lrq_ordered_float(slot[0]), b = lrq_ordered_float(slot[1]);
+                t = token_params_fast(a, b, A_BITS, mode, 1.0 / sqrt((double)(1 << LOG2B)), &sc, &z);
+                if (j == 0 && live) { scale[m] = sc; zp[m] = z; }
+            }
+            t.inv = __shfl_sync(seg_mask, t.inv, seg_lane);
+            t.negz = __shfl_sync(seg_mask, t.negz, seg_lane);
+        }
+        if (tid < 2 * tok_per_cta) ext[((it + 2) % 3) * 2 * tok_per_cta + tid] = (tid & 1) ? INT_MIN : INT_MAX;
+        if (live) {
+            const f32x2 INV = pack2(t.inv, t.inv), NEGZ = pack2(t.negz, t.negz);
+            // run r holds elements r * (B / 4) + 8 * tau .. + 7 of the thread's transform block
+            const size_t e0 = (size_t)m * K + (size_t)unit_in_token * (U * 1024) + (size_t)tau * 8;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                int q[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float x, y;
+                    unpack2(fma2(P[4 * r + i], INV, NEGZ), x, y);
+                    q[2 * i] = __float2int_rn(x); q[2 * i + 1] = __float2int_rn(y);
+                }
+                const size_t e = e0 + (size_t)r * (U * 256);
+                if (A_BITS == 8) {
+                    *reinterpret_cast<uint2*>(codes + e) = make_uint2(pack_u8x4(q[0], q[1], q[2], q[3]), pack_u8x4(q[4], q[5], q[6], q[7]));
+                } else {
+                    *reinterpret_cast<uint32_t*>(codes + (e >> 1)) = pack_u4x8(q);
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Quantizer of already rotated fp32 rows whose extremes are known (dense path: the rotation GEMM's epilogue
 // found them).  One warp per token, grid-stride; lane 0 works out the step and zero-point, then the warp
 // streams the row: 32 bytes in (one 256-bit load), 8 or 4 code bytes out per lane and step.
@@ -566,7 +757,16 @@ static lrq_status launch_generic(bool f32, const void* X, int M, int K, long ldx
     return LRQ_OK;
 }
 
-template <int LOG2B>
+template <int LOG2B, bool BIG, int A_BITS, int NT, int NB, bool WIDE>
+struct RotqPick {
+    static constexpr auto kern = rotq_fast_kernel<LOG2B, A_BITS, NT, NB, WIDE>;
+};
+template <int LOG2B, int A_BITS, int NT, int NB, bool WIDE>
+struct RotqPick<LOG2B, true, A_BITS, NT, NB, WIDE> {
+    static constexpr auto kern = rotq_big_kernel<LOG2B, A_BITS, NT, NB, WIDE>;
+};
+
+template <int LOG2B, bool BIG = false>
 static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits, int mode, const float* prescale, uint8_t* codes,
                               float* scale, int32_t* zp, cudaStream_t st) {
     const int tpt = K / EPT;
@@ -577,15 +777,20 @@ static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits,
     while (T * tpt < 256 && (T + T0) * tpt <= 512) T += T0;
     const int threads = T * tpt;
     if (threads > 512) return LRQ_ERR_UNSUPPORTED;
-    size_t smem = 3 * 2 * sizeof(int) * T + 16;
-    if (LOG2B > 10) smem += (size_t)threads * EPT * sizeof(float);
+    size_t smem = 3 * 2 * sizeof(int) * T + (BIG ? 128 : 16);
+    if (BIG) {                                       // one buffer of B + 32 floats per transform block held by the CTA
+        const int B = 1 << LOG2B;
+        smem += (size_t)(threads * EPT / B) * (size_t)(B + 32) * sizeof(float);
+    } else if (LOG2B > 10) {
+        smem += (size_t)threads * EPT * sizeof(float);
+    }
     // register budget by CTA size: three CTAs of up to 288 threads, two of up to 384, else one
     typedef void (*Kern)(const __nv_bfloat16*, int, int, long, int, int, int, const float*, uint8_t*, float*, int32_t*);
     // 256-bit accesses when every thread's 64 input bytes and 32 code bytes start on 32-byte boundaries
     const bool wide = lrq_aligned(X, 32) && (ldx % 16) == 0 && lrq_aligned(codes, 32);
     Kern kern;
-#define LRQ_PICK(NT, NB) (wide ? (a_bits == 8 ? rotq_fast_kernel<LOG2B, 8, NT, NB, true> : rotq_fast_kernel<LOG2B, 4, NT, NB, true>) \
-                               : (a_bits == 8 ? rotq_fast_kernel<LOG2B, 8, NT, NB, false> : rotq_fast_kernel<LOG2B, 4, NT, NB, false>))
+#define LRQ_PICK(NT, NB) (wide ? (a_bits == 8 ? RotqPick<LOG2B, BIG, 8, NT, NB, true>::kern : RotqPick<LOG2B, BIG, 4, NT, NB, true>::kern) \
+                               : (a_bits == 8 ? RotqPick<LOG2B, BIG, 8, NT, NB, false>::kern : RotqPick<LOG2B, BIG, 4, NT, NB, false>::kern))
     if (threads <= 288) kern = LRQ_PICK(288, 3);
     else if (threads <= 384) kern = LRQ_PICK(384, 2);
     else kern = LRQ_PICK(512, 1);
@@ -614,8 +819,10 @@ lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B
         lrq_status r = LRQ_ERR_UNSUPPORTED;
         switch (log2B) {
 #define LRQ_CASE(L) case L: r = launch_fast<L>(X, M, K, ldx, a_bits, mode, prescale, codes, scale, zp, st); break;
-            LRQ_CASE(3) LRQ_CASE(4) LRQ_CASE(5) LRQ_CASE(6) LRQ_CASE(7) LRQ_CASE(8) LRQ_CASE(9) LRQ_CASE(10)
-            LRQ_CASE(11) LRQ_CASE(12)
+            LRQ_CASE(3) LRQ_CASE(4) LRQ_CASE(5) LRQ_CASE(6) LRQ_CASE(7) LRQ_CASE(8) LRQ_CASE(9)
+#undef LRQ_CASE
+#define LRQ_CASE(L) case L: r = launch_fast<L, true>(X, M, K, ldx, a_bits, mode, prescale, codes, scale, zp, st); break;
+            LRQ_CASE(10) LRQ_CASE(11) LRQ_CASE(12)
 #undef LRQ_CASE
             default: break;
         }
