@@ -158,9 +158,9 @@ rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log
 // ------------------------------------------------------------------------------------------------
 // Fast kernel.  A thread owns 32 consecutive elements of one token (four 128-bit loads in flight,
 // the next token group's loads issued before the current group's arithmetic): index bits 0-4 of the
-// transform are butterflies between its own registers, bits 5-9 are butterflies with the lane whose
-// index differs in one bit (two shuffles and one packed fused multiply-add per element pair and
-// stage), bits 10-11 (B = 2048, 4096) go through shared memory.  All fp32 arithmetic on element
+// transform are butterflies between its own registers, bits 5-8 (B up to 512) are butterflies with the
+// lane whose index differs in one bit (two shuffles and one packed fused multiply-add per element pair
+// and stage); larger blocks take rotq_big_kernel below.  All fp32 arithmetic on element
 // pairs uses the packed two-wide instructions (add/sub/fma.f32x2): one issue slot per two elements.
 // A CTA holds T whole tokens (T * K/32 threads, a multiple of 32) and walks over token groups with
 // a grid stride; the token's extremes are reduced through shared memory, then every thread
@@ -317,9 +317,9 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
 #pragma unroll
             for (int i = 0; i < NP; ++i)
                 if (!(i & h)) { const f32x2 a = P[i], b = P[i | h]; P[i] = add2(a, b); P[i | h] = sub2(a, b); }
-        // index bits 5..9: partner lanes
+        // index bits 5..8: partner lanes
 #pragma unroll
-        for (int b = 5; b < LOG2B && b < 10; ++b) {
+        for (int b = 5; b < LOG2B; ++b) {
             const int lm = 1 << (b - 5);
             const float sg = (lane & lm) ? -1.f : 1.f;
             const f32x2 S = pack2(sg, sg);
@@ -329,28 +329,6 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
                 unpack2(P[i], x, y);
                 const float ox = __shfl_xor_sync(0xffffffffu, x, lm), oy = __shfl_xor_sync(0xffffffffu, y, lm);
                 P[i] = fma2(P[i], S, pack2(ox, oy));     // low lane: own + other, high lane: other - own
-            }
-        }
-        // index bits 10..11: partner warps, through shared memory (chunk index swizzled by the lane)
-        if (LOG2B > 10) {
-            ulonglong2* xb = reinterpret_cast<ulonglong2*>(ext + 3 * 2 * tok_per_cta);
-            xb = reinterpret_cast<ulonglong2*>((reinterpret_cast<uintptr_t>(xb) + 15) & ~uintptr_t(15));
-#pragma unroll
-            for (int b = 10; b < LOG2B; ++b) {
-                const int tm = 1 << (b - 5);
-                __syncthreads();
-#pragma unroll
-                for (int c = 0; c < 8; ++c) xb[tid * 8 + (c ^ (lane & 7))] = make_ulonglong2(P[2 * c], P[2 * c + 1]);
-                __syncthreads();
-                const int pt = tid ^ tm;
-                const float sg = (tid & tm) ? -1.f : 1.f;
-                const f32x2 S = pack2(sg, sg);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const ulonglong2 o = xb[pt * 8 + (c ^ (lane & 7))];
-                    P[2 * c] = fma2(P[2 * c], S, o.x);
-                    P[2 * c + 1] = fma2(P[2 * c + 1], S, o.y);
-                }
             }
         }
         // extremes of the thread's values, of the token's lanes in this warp (one redux each on order-preserving
@@ -781,8 +759,6 @@ static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits,
     if (BIG) {                                       // one buffer of B + 32 floats per transform block held by the CTA
         const int B = 1 << LOG2B;
         smem += (size_t)(threads * EPT / B) * (size_t)(B + 32) * sizeof(float);
-    } else if (LOG2B > 10) {
-        smem += (size_t)threads * EPT * sizeof(float);
     }
     // register budget by CTA size: three CTAs of up to 288 threads, two of up to 384, else one
     typedef void (*Kern)(const __nv_bfloat16*, int, int, long, int, int, int, const float*, uint8_t*, float*, int32_t*);
