@@ -27,6 +27,8 @@ def P():
     (1, 128, 128, 8, 0), (7, 1152, 128, 8, 0), (129, 1024, 1024, 4, 0), (33, 1536, 512, 4, 0),
     (5, 6144, 2048, 4, 0), (3, 12288, 4096, 4, 0), (17, 3072, 1024, 4, 1), (64, 4608, 128, 8, 1),
     (9, 64, 8, 8, 0), (12, 256, 16, 4, 0), (300, 1152, 128, 4, 0), (2, 512, 64, 8, 0),
+    # large blocks (register-butterfly kernel): 8-bit codes, several blocks per token, several groups per CTA
+    (4001, 1024, 1024, 8, 0), (70, 2048, 2048, 8, 0), (130, 8192, 4096, 8, 1), (257, 2048, 1024, 4, 0),
 ])
 def test_rotate_quantize_hadamard(P, orc, M, K, B, a_bits, mode):
     xb = make_activations(100 + M + K, M, K)
