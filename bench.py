@@ -37,12 +37,12 @@ from lrq_workloads import bf16_bits_to_f64, config_layers, default_clip_grid  # 
 # profiles/, keyed by the kernel and layer the roofline object describes.  A key is dropped (traffic: null) when its
 # kernel changes after the capture.
 NCU_TRAFFIC_BYTES = {
-    "qgemm cfg1 fc1": 7.76e6 + 17.17e6,
-    "qgemm cfg3 fc1": 27.11e6 + 168.94e6,
-    "qgemm cfg4 b0.fc1": 219.61e6 + 553.28e6,
+    "qgemm cfg1 fc1": 7.77e6 + 19.03e6,
+    "qgemm cfg3 fc1": 27.04e6 + 170.13e6,
+    "qgemm cfg4 b0.fc1": 234.89e6 + 553.87e6,
     "rotq cfg1 fc2": None,                      # 57 MB case not captured; the M = 32768 capture of the same layer shape:
-    "rotq cfg4 b0.fc2": 302.30e6 + 122.04e6,
-    "rotq cfg3 fc2": 113.29e6 + 11.98e6,
+    "rotq cfg4 b0.fc2": 302.21e6 + 122.65e6,
+    "rotq cfg3 fc2": 113.27e6 + 12.87e6,
 }
 
 METRIC = "qlinear_tflops"
