@@ -1,4 +1,4 @@
-"""GPU parity at the BASELINE workload sizes, in the launch configuration the bench times: every layer is
+"""GPU parity at the full workload sizes, in the launch configuration the bench times: every layer is
 run in full through lrq_qlinear; activation codes are compared for all tokens where the oracle's rotation is
 cheap (Hadamard) and for sampled tokens otherwise; outputs are compared on sampled token rows; TLQ codes and
 tables on sampled weight rows."""

@@ -1,6 +1,6 @@
 """GPU parity: every step of the CUDA path, called through the C ABI, against the fp64 oracle on the same
 seeded inputs.  Small shapes are compared element by element (several tiles plus a ragged tail); the
-BASELINE-sized layers are run in full on the GPU and compared on sampled token rows, which the oracle
+full-size workload layers are run in full on the GPU and compared on sampled token rows, which the oracle
 computes one by one (tokens are independent)."""
 import numpy as np
 import pytest
@@ -192,7 +192,7 @@ def test_qlinear_stack_matches_single_calls(P):
 @pytest.mark.parametrize("cfg,li", [(1, 0), (2, 0), (3, 1)])
 def test_qgemm_tensor_core_matches_cuda_core_everywhere(P, cfg, li):
     # Every output element of the tcgen05 kernel against the plain CUDA-core kernel of the same library on a
-    # BASELINE-sized layer: several tiles per CTA pair, grouped and per-channel tables, 4- and 8-bit codes.
+    # full-size workload layer: several tiles per CTA pair, grouped and per-channel tables, 4- and 8-bit codes.
     # The oracle checks sampled rows elsewhere; this one looks at all of them, twice (a hand-over race
     # between the kernel's warps shows up as a few wrong tiles that differ from run to run).
     spec = config_layers(cfg)[li]
