@@ -46,6 +46,12 @@ typedef enum {
 typedef enum { LRQ_ROT_NONE = 0, LRQ_ROT_HADAMARD = 1, LRQ_ROT_DENSE = 2 } lrq_rot_kind;
 typedef enum { LRQ_ACT_ASYM = 0, LRQ_ACT_SYM = 1 } lrq_act_mode;
 typedef enum { LRQ_F32 = 0, LRQ_F16 = 1, LRQ_BF16 = 2 } lrq_dtype;
+/* Storage of the weight codes (Sec. 4.1, Eq. 5: a b-bit code per weight).
+ *   NIBBLE   two codes per byte, element 2j in the low nibble of byte j; row pitch K/2 bytes (b = 2..4)
+ *   PACKED3  b = 3 only: eight codes in three bytes, code j of each eight at bits 3j..3j+2 of the little-endian
+ *            24-bit word; row pitch 3K/8 bytes.  The storage TLQ's 3-bit codes actually need; taken by the
+ *            weight-bandwidth-bound contraction for small token counts. */
+typedef enum { LRQ_CODES_NIBBLE = 0, LRQ_CODES_PACKED3 = 1 } lrq_code_layout;
 
 /* ---------------------------------------------------------------------------------------------
  * TLQ weight quantization (Sec. 4.1: Eqs. 4-5 twin-log quantizer, Eq. 6 search-based clipping,
@@ -53,8 +59,8 @@ typedef enum { LRQ_F32 = 0, LRQ_F16 = 1, LRQ_BF16 = 2 } lrq_dtype;
  *
  * For every output row n and every group of `group_size` consecutive input channels the kernel
  * takes log2|w| of the positive and of the negative elements separately, searches the clipping
- * factor of each side over the caller's grid (squared error of the de-quantized magnitudes,
- * first minimum wins), and emits the signed code of Eq. 5 plus the table of level values
+ * factor of each side over the caller's grid (squared error of the de-quantized magnitudes, summed in
+ * fp64 over the side's elements in increasing k; first minimum in grid order wins), and emits the signed code of Eq. 5 plus the table of level values
  * II * 2^(f-I) of Eqs. 8-9.  Code 0 is shared by the lowest positive level, by negative elements
  * that round to the negative side's code 0, and by exact zeros; its table entry is the lowest
  * positive level.
@@ -66,11 +72,12 @@ typedef struct {
     int n_alpha, n_beta;   /* grid sizes, 1..64                                                   */
     const double* alpha;   /* host: clipping factors tried on the positive side (Eq. 6)          */
     const double* beta;    /* host: clipping factors tried on the negative side                  */
+    lrq_code_layout code_layout;   /* how `codes` is written; PACKED3 needs w_bits == 3                    */
 } lrq_tlq_params;
 
 /*
  * W_rot  dev  float [N,K]   weights in the rotated basis (W.R of Eq. 2), row-major, 16-byte aligned
- * codes  dev  uint8 [N,K/2] packed offset-binary codes (out)
+ * codes  dev  uint8 [N,K/2] (NIBBLE) or [N,3K/8] (PACKED3) offset-binary codes u = c + 2^(b-1) (out)
  * levels dev  float [N,K/G,2^b] level tables (out)
  * meta   dev  double [N,K/G,6]  s+, z+, s-, z-, alpha, beta chosen per group (out, may be NULL)
  * wsum   dev  float [N]     sum over k of the de-quantized row, used by the zero-point term (out)
@@ -180,12 +187,13 @@ lrq_status lrq_rotate_quantize_act_static(const void* X_bf16, int M, int K, long
  * A quantized layer: TLQ codes, level tables and the activation recipe of one linear.
  * The handle is a small host object; it stores the device pointers it is given (it does not
  * copy or own them) and must be destroyed with lrq_layer_destroy.
- *   codes [N,K/2], levels [N,K/G,2^b], wsum [N] as produced by lrq_tlq_quantize_weights;
+ *   codes [N,K/2] or [N,3K/8] (code_layout), levels [N,K/G,2^b], wsum [N] as produced by
+ *   lrq_tlq_quantize_weights (codes, levels 16-byte aligned);
  *   wscale (nullable) float [N] per-channel output scale, bias (nullable) float [N].
  * ------------------------------------------------------------------------------------------- */
 typedef struct lrq_layer lrq_layer;
 
-lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size,
+lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size, lrq_code_layout code_layout,
                             const uint8_t* codes, const float* levels, const float* wsum,
                             const float* wscale, const float* bias, const lrq_act_params* act);
 void lrq_layer_destroy(lrq_layer* L);
@@ -222,6 +230,14 @@ lrq_status lrq_qgemm_codes(const lrq_layer* L, const uint8_t* a_codes, const flo
 /* Code recorded by a bounded device-side wait that expired since the last call of this function
  * (0 if none).  Synchronises `cuda_stream` to read it. */
 int lrq_device_status(void* cuda_stream);
+
+/* Diagnostic of the bounded waits (no counterpart in the paper): launches a one-warp kernel that waits, through the
+ * same bounded-wait routine the tensor-core kernels use, on a barrier nothing ever arrives on.  After
+ * `limit_cycles` SM clock cycles (1 .. 1e8) the wait gives up, records LRQ_SELFTEST_WAIT_CODE in the status word
+ * and the kernel returns; lrq_device_status() then reports that code once.  Nothing else is in flight in that
+ * kernel, so the context stays usable. */
+#define LRQ_SELFTEST_WAIT_CODE 99
+lrq_status lrq_selftest_wait_timeout(long long limit_cycles, void* cuda_stream);
 
 const char* lrq_status_string(lrq_status s);
 int lrq_version(void);

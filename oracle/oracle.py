@@ -224,9 +224,10 @@ def qmatmul(Q, S, Z, tlq: TLQResult, wscale=None, bias=None):
 
 
 def qlinear(X, tlq: TLQResult, a_bits: int, rot: str, had_block: int = 0, R=None, mode: int = 0,
-            wscale=None, bias=None, prescale=None):
+            wscale=None, bias=None, prescale=None, return_rotated: bool = False):
     """The whole layer on already-widened inputs: [smooth (Sec. 5.1) ->] rotate (Eq. 12) -> per-token
-    quantize (Eq. 1) -> contraction with the TLQ table and epilogue (Eq. 10).  Returns (Y, codes, s, z)."""
+    quantize (Eq. 1) -> contraction with the TLQ table and epilogue (Eq. 10).  Returns (Y, codes, s, z), and with
+    return_rotated also the rotated activations that Eq. 1 quantized."""
     if prescale is not None:
         X = smooth(X, prescale)
     if rot == "hadamard":
@@ -238,4 +239,5 @@ def qlinear(X, tlq: TLQResult, a_bits: int, rot: str, had_block: int = 0, R=None
     else:
         raise ValueError(rot)
     Q, S, Z = quantize_act(Yr, a_bits, mode)
-    return qmatmul(Q, S, Z, tlq, wscale, bias), Q, S, Z
+    Y = qmatmul(Q, S, Z, tlq, wscale, bias)
+    return (Y, Q, S, Z, Yr) if return_rotated else (Y, Q, S, Z)

@@ -15,13 +15,14 @@ _LIBPATH = os.path.join(_HERE, "liblrq_b200.so")
 ROT_NONE, ROT_HADAMARD, ROT_DENSE = 0, 1, 2
 ACT_ASYM, ACT_SYM = 0, 1
 F32, F16, BF16 = 0, 1, 2
+CODES_NIBBLE, CODES_PACKED3 = 0, 1
 _TORCH_DT = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16}
 
 EXPORTS = [
     "lrq_tlq_quantize_weights", "lrq_act_workspace_bytes", "lrq_rotate_quantize_act", "lrq_layer_create",
     "lrq_layer_destroy", "lrq_workspace_bytes", "lrq_qlinear", "lrq_qlinear_stack", "lrq_qgemm_codes",
     "lrq_device_status", "lrq_status_string", "lrq_version", "lrq_rotate_quantize_act_static", "lrq_ars_select",
-    "lrq_rotate_weights",
+    "lrq_rotate_weights", "lrq_selftest_wait_timeout",
 ]
 STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -36,7 +37,7 @@ class LrqError(RuntimeError):
 class _TlqParams(C.Structure):
     _fields_ = [("w_bits", C.c_int), ("group_size", C.c_int), ("integerize_I", C.c_int),
                 ("n_alpha", C.c_int), ("n_beta", C.c_int),
-                ("alpha", C.POINTER(C.c_double)), ("beta", C.POINTER(C.c_double))]
+                ("alpha", C.POINTER(C.c_double)), ("beta", C.POINTER(C.c_double)), ("code_layout", C.c_int)]
 
 
 class _ActParams(C.Structure):
@@ -63,7 +64,7 @@ def load_library() -> C.CDLL:
     lib.lrq_act_workspace_bytes.restype = sz
     lib.lrq_rotate_quantize_act.argtypes = [vp, ci, ci, cl, C.POINTER(_ActParams), vp, vp, vp, vp, sz, vp]
     lib.lrq_rotate_quantize_act_static.argtypes = [vp, ci, ci, cl, C.POINTER(_ActParams), vp, vp, vp, vp]
-    lib.lrq_layer_create.argtypes = [C.POINTER(vp), ci, ci, ci, ci, vp, vp, vp, vp, vp, C.POINTER(_ActParams)]
+    lib.lrq_layer_create.argtypes = [C.POINTER(vp), ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, C.POINTER(_ActParams)]
     lib.lrq_layer_destroy.argtypes = [vp]
     lib.lrq_layer_destroy.restype = None
     lib.lrq_workspace_bytes.argtypes = [vp, ci]
@@ -75,6 +76,7 @@ def load_library() -> C.CDLL:
     lib.lrq_ars_select.argtypes = [vp, ci, ci, cl, C.c_double, vp, vp, vp, sz, vp]
     lib.lrq_rotate_weights.argtypes = [vp, ci, ci, cl, vp, ci, ci, vp, vp, cl, vp]
     lib.lrq_device_status.argtypes = [vp]
+    lib.lrq_selftest_wait_timeout.argtypes = [C.c_longlong, vp]
     lib.lrq_status_string.argtypes = [ci]
     lib.lrq_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -112,38 +114,47 @@ def lrq_device_status(stream=None) -> int:
     return int(load_library().lrq_device_status(_stream(stream)))
 
 
+def lrq_selftest_wait_timeout(limit_cycles: int = 100000, stream=None) -> None:
+    """Launch the diagnostic kernel whose bounded wait runs out; lrq_device_status() then returns SELFTEST_WAIT_CODE once."""
+    _check(load_library().lrq_selftest_wait_timeout(int(limit_cycles), _stream(stream)), "lrq_selftest_wait_timeout")
+
+
+SELFTEST_WAIT_CODE = 99
+
+
 # ------------------------------------------------------------------------------------------------
 @dataclass
 class TLQWeights:
-    codes: torch.Tensor    # uint8 [N, K/2]
+    codes: torch.Tensor    # uint8 [N, K/2] (nibbles) or [N, 3K/8] (packed 3-bit)
     levels: torch.Tensor   # float32 [N, K/G, 2^b]
     meta: torch.Tensor     # float64 [N, K/G, 6]
     wsum: torch.Tensor     # float32 [N]
     w_bits: int
     group: int             # 0 = per output channel
+    code_layout: int = CODES_NIBBLE
 
 
 def lrq_tlq_quantize_weights(W_rot: torch.Tensor, w_bits: int, group_size: int = 0, integerize_I: int = 7,
                              alpha: Sequence[float] = (1.0,), beta: Sequence[float] = (1.0,),
-                             stream=None) -> TLQWeights:
+                             stream=None, code_layout: int = CODES_NIBBLE) -> TLQWeights:
     """TLQ weight quantization (Sec. 4.1, Eqs. 4-9) of a device float32 [N,K] matrix."""
     _need_cuda(W_rot)
     assert W_rot.dtype == torch.float32 and W_rot.is_contiguous() and W_rot.dim() == 2
     N, K = W_rot.shape
     G = K if group_size <= 0 else group_size
     dev = W_rot.device
-    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+    codes = torch.empty((N, 3 * K // 8 if code_layout == CODES_PACKED3 else K // 2), dtype=torch.uint8, device=dev)
     levels = torch.empty((N, max(1, K // max(G, 1)), 1 << w_bits), dtype=torch.float32, device=dev)
     meta = torch.empty((N, max(1, K // max(G, 1)), 6), dtype=torch.float64, device=dev)
     wsum = torch.empty((N,), dtype=torch.float32, device=dev)
     a = (C.c_double * len(alpha))(*[float(v) for v in alpha])
     b = (C.c_double * len(beta))(*[float(v) for v in beta])
     p = _TlqParams(int(w_bits), int(group_size), int(integerize_I), len(alpha), len(beta),
-                   C.cast(a, C.POINTER(C.c_double)), C.cast(b, C.POINTER(C.c_double)))
+                   C.cast(a, C.POINTER(C.c_double)), C.cast(b, C.POINTER(C.c_double)), int(code_layout))
     rc = load_library().lrq_tlq_quantize_weights(_ptr(W_rot), N, K, C.byref(p), _ptr(codes), _ptr(levels),
                                                  _ptr(meta), _ptr(wsum), None, 0, _stream(stream))
     _check(rc, "lrq_tlq_quantize_weights")
-    return TLQWeights(codes, levels, meta, wsum, int(w_bits), int(group_size))
+    return TLQWeights(codes, levels, meta, wsum, int(w_bits), int(group_size), int(code_layout))
 
 
 def _act_params(kind: int, had_block: int, R: Optional[torch.Tensor], a_bits: int, mode: int,
@@ -252,7 +263,7 @@ class QLayer:
         self.kind, self.a_bits, self.had_block, self.mode = kind, a_bits, had_block, mode
         self._p = _act_params(kind, had_block, R, a_bits, mode, prescale)
         h = C.c_void_p()
-        rc = load_library().lrq_layer_create(C.byref(h), N, K, tlq.w_bits, tlq.group, _ptr(tlq.codes),
+        rc = load_library().lrq_layer_create(C.byref(h), N, K, tlq.w_bits, tlq.group, tlq.code_layout, _ptr(tlq.codes),
                                              _ptr(tlq.levels), _ptr(tlq.wsum), _ptr(wscale), _ptr(bias),
                                              C.byref(self._p))
         _check(rc, "lrq_layer_create")

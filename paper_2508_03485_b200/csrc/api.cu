@@ -18,6 +18,30 @@ int* lrq_status_word() {
     return p;
 }
 
+// Current device and its SM count.  The attribute is queried once per device; the cache is filled under a
+// lock and read-only afterwards.
+lrq_status lrq_current_device(int* dev_out, int* sms_out) {
+    static std::mutex mu;
+    static int sms_of[LRQ_MAX_DEVICES] = {};
+    int dev = -1;
+    LRQ_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= LRQ_MAX_DEVICES) return LRQ_ERR_UNSUPPORTED;
+    int sms;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!sms_of[dev]) {
+            int v = 0;
+            LRQ_CUDA_TRY(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev));
+            if (v < 1) return LRQ_ERR_CUDA;
+            sms_of[dev] = v;
+        }
+        sms = sms_of[dev];
+    }
+    if (dev_out) *dev_out = dev;
+    if (sms_out) *sms_out = sms;
+    return LRQ_OK;
+}
+
 static lrq_status check_act(const lrq_act_params* p, int K) {
     if (!p) return LRQ_ERR_INVALID_ARG;
     if (p->a_bits != 4 && p->a_bits != 8) return LRQ_ERR_UNSUPPORTED;
@@ -59,12 +83,9 @@ extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long 
         float* Yr = static_cast<float*>(workspace);
         // the rotation leaves each token's extremes in the scale / zero-point outputs (as integers); the
         // quantizer reads them and then writes the real values there
-        bool have_ext = false;
-        st = lrq_launch_rotgemm(X, M, K, ldx, p->R_bf16, Yr, reinterpret_cast<int*>(a_scale), reinterpret_cast<int*>(a_zp),
-                                &have_ext, stream);
+        st = lrq_launch_rotgemm(X, M, K, ldx, p->R_bf16, Yr, reinterpret_cast<int*>(a_scale), reinterpret_cast<int*>(a_zp), stream);
         if (st != LRQ_OK) return st;
-        if (have_ext) return lrq_launch_quantize_f32_ext(Yr, M, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
-        return lrq_launch_quantize_f32(Yr, M, K, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
+        return lrq_launch_quantize_f32_ext(Yr, M, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
     }
     const int B = p->kind == LRQ_ROT_HADAMARD ? p->had_block : 1;
     return lrq_launch_rotq_hadamard(X, M, K, ldx, B, p->a_bits, p->mode, p->prescale, a_codes, a_scale, a_zp, stream);
@@ -134,12 +155,14 @@ extern "C" lrq_status lrq_rotate_weights(const float* W, int N, int K, long ldw,
 }
 
 extern "C" lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size,
-                                       const uint8_t* codes, const float* levels, const float* wsum,
+                                       lrq_code_layout code_layout, const uint8_t* codes, const float* levels, const float* wsum,
                                        const float* wscale, const float* bias, const lrq_act_params* act) {
     if (!out) return LRQ_ERR_INVALID_ARG;
     *out = nullptr;
     if (!codes || !levels || !wsum || N <= 0 || K <= 0) return LRQ_ERR_INVALID_ARG;
     if (w_bits < 2 || w_bits > 4) return LRQ_ERR_UNSUPPORTED;
+    if (code_layout != LRQ_CODES_NIBBLE && code_layout != LRQ_CODES_PACKED3) return LRQ_ERR_INVALID_ARG;
+    if (code_layout == LRQ_CODES_PACKED3 && w_bits != 3) return LRQ_ERR_UNSUPPORTED;
     const int G = group_size > 0 ? group_size : K;
     if (K % G || G % 8) return LRQ_ERR_UNSUPPORTED;
     lrq_status st = check_act(act, K);
@@ -147,9 +170,11 @@ extern "C" lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits
     if (!lrq_aligned(codes, 16) || !lrq_aligned(levels, 16)) return LRQ_ERR_INVALID_ARG;
     lrq_layer* L = new (std::nothrow) lrq_layer;
     if (!L) return LRQ_ERR_INVALID_ARG;
-    L->N = N; L->K = K; L->w_bits = w_bits; L->group = G;
+    L->N = N; L->K = K; L->w_bits = w_bits; L->group = G; L->packed3 = code_layout == LRQ_CODES_PACKED3 ? 1 : 0;
     L->codes = codes; L->levels = levels; L->wsum = wsum; L->wscale = wscale; L->bias = bias;
     L->act = *act;
+    L->have_tm_w = false;
+    lrq_qgemm_tc_prepare(L);          // caches the weight-code TMA descriptors when the shape takes that kernel
     *out = L;
     return LRQ_OK;
 }
@@ -204,13 +229,22 @@ extern "C" lrq_status lrq_qgemm_codes(const lrq_layer* L, const uint8_t* a_codes
     return qgemm_dispatch(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, impl, (cudaStream_t)cuda_stream);
 }
 
-extern "C" lrq_status lrq_qlinear(const lrq_layer* L, const void* X, int M, long ldx, void* Y, lrq_dtype dt, long ldy,
-                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+// Every check lrq_qlinear makes on one layer's arguments; nothing is launched here.
+static lrq_status validate_layer_call(const lrq_layer* L, const void* X, int M, long ldx, const void* Y, lrq_dtype dt,
+                                      long ldy, const void* workspace, size_t workspace_bytes) {
     if (!L || !X || M <= 0) return LRQ_ERR_INVALID_ARG;
     lrq_status st = check_out(Y, dt, ldy, L->N);
     if (st != LRQ_OK) return st;
+    if (ldx < L->K || (ldx % 8) || !lrq_aligned(X, 16)) return LRQ_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < ws_layout(L, M).total || !lrq_aligned(workspace, 256)) return LRQ_ERR_WORKSPACE;
+    return LRQ_OK;
+}
+
+extern "C" lrq_status lrq_qlinear(const lrq_layer* L, const void* X, int M, long ldx, void* Y, lrq_dtype dt, long ldy,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    lrq_status st = validate_layer_call(L, X, M, ldx, Y, dt, ldy, workspace, workspace_bytes);
+    if (st != LRQ_OK) return st;
     const WsLayout w = ws_layout(L, M);
-    if (!workspace || workspace_bytes < w.total || !lrq_aligned(workspace, 256)) return LRQ_ERR_WORKSPACE;
     char* base = static_cast<char*>(workspace);
     uint8_t* a_codes = reinterpret_cast<uint8_t*>(base + w.codes);
     float* a_scale = reinterpret_cast<float*>(base + w.scale);
@@ -226,12 +260,10 @@ extern "C" lrq_status lrq_qlinear_stack(const lrq_layer* const* layers, int n_la
                                         const long* ldy, void* workspace, size_t workspace_bytes,
                                         void* cuda_stream) {
     if (!layers || !X || !M || !ldx || !Y || !ldy || n_layers <= 0) return LRQ_ERR_INVALID_ARG;
-    // validate everything before the first launch
+    // every layer's arguments are validated before the first launch
     for (int i = 0; i < n_layers; ++i) {
-        if (!layers[i] || !X[i] || M[i] <= 0) return LRQ_ERR_INVALID_ARG;
-        lrq_status st = check_out(Y[i], dt, ldy[i], layers[i]->N);
+        lrq_status st = validate_layer_call(layers[i], X[i], M[i], ldx[i], Y[i], dt, ldy[i], workspace, workspace_bytes);
         if (st != LRQ_OK) return st;
-        if (!workspace || workspace_bytes < lrq_workspace_bytes(layers[i], M[i])) return LRQ_ERR_WORKSPACE;
     }
     for (int i = 0; i < n_layers; ++i) {
         lrq_status st = lrq_qlinear(layers[i], X[i], M[i], ldx[i], Y[i], dt, ldy[i], workspace, workspace_bytes,

@@ -35,7 +35,9 @@
 // accumulator free of a large common-mode term.
 #include "lrq_internal.cuh"
 #include "tc_ptx.cuh"
+#include "f32x2.cuh"
 #include "tma_host.cuh"
+#include <mutex>
 
 namespace {
 using namespace lrq_tc;
@@ -209,12 +211,7 @@ struct RingPos {
 };
 static_assert(STAGES % 2 == 0 && CSTAGES % 2 == 0, "the two decode groups own alternate ring slots");
 
-typedef unsigned long long f32x2;      // two fp32 values in one 64-bit register pair
-__device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
-__device__ __forceinline__ void unpack2(f32x2 r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+using namespace lrq_f2;
 
 struct Params {
     const float* a_scale; const int32_t* a_zp;
@@ -272,6 +269,10 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
     cluster_sync_all();                       // the peer's barriers exist before anyone arrives on them
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    // everything above touched no global memory: it may overlap the tail of the kernel before this one in the
+    // stream (which produced the activation codes); everything below must see that kernel's writes
+    lrq_pdl_trigger();
+    lrq_pdl_wait();
 
     if (warp == TMA_WARP) {
         // =============================== packed codes: global -> shared (TMA) ===============================
@@ -613,22 +614,33 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
 template <int A_BITS, int W_BITS, int BN_T>
 lrq_status launch(const Params& p, const CUtensorMap& tmA, const CUtensorMap& tmW, const CUtensorMap& tmY, int num_tiles, cudaStream_t st) {
     auto kern = qgemm_tc_kernel<A_BITS, W_BITS, BN_T>;
-    static int max_pairs = 0;                 // per process; the library targets identical GPUs
+    // per device and kernel variant: the shared-memory opt-in (a per-device function attribute) and the number of
+    // CTA pairs that can be resident; set up once under a lock, read-only afterwards
+    static std::mutex mu;
+    static int max_pairs_of[LRQ_MAX_DEVICES] = {};
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(NUM_THREADS); cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    if (!max_pairs) {
-        LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-        int dev = 0, sms = 0, clusters = 0;
-        LRQ_CUDA_TRY(cudaGetDevice(&dev));
-        LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        cfg.gridDim = dim3(sms & ~1);
-        LRQ_CUDA_TRY(cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg));
-        if (clusters < 1) return LRQ_ERR_CUDA;
-        max_pairs = clusters < sms / 2 ? clusters : sms / 2;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    int dev = 0, sms = 0, max_pairs = 0;
+    if (lrq_current_device(&dev, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!max_pairs_of[dev]) {
+            LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+            int clusters = 0;
+            cfg.gridDim = dim3(sms & ~1);
+            cfg.numAttrs = 1;                 // the occupancy query looks at the cluster shape only
+            LRQ_CUDA_TRY(cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg));
+            cfg.numAttrs = 2;
+            if (clusters < 1) return LRQ_ERR_CUDA;
+            max_pairs_of[dev] = clusters < sms / 2 ? clusters : sms / 2;
+        }
+        max_pairs = max_pairs_of[dev];
     }
     const int pairs = num_tiles < max_pairs ? num_tiles : max_pairs;
     cfg.gridDim = dim3(2 * pairs);
@@ -636,14 +648,42 @@ lrq_status launch(const Params& p, const CUtensorMap& tmA, const CUtensorMap& tm
     return LRQ_OK;
 }
 
+// Tile width.  A 128-wide tile was measured at about 0.87 of the time of a 256-wide one (the weight decode
+// halves; the activation expansion, the hand-overs and the epilogue set-up do not), so it only pays when it
+// cuts the number of rounds of tiles over the CTA pairs: small M with a narrow or ragged N (80 wide tiles on
+// 74 pairs are two rounds, the same work as 144 narrow tiles is two cheaper rounds).
+bool narrow_tiles(int M, int N, int sms, long* tiles) {
+    const long pairs_avail = sms / 2 > 0 ? sms / 2 : 1;
+    const long tiles_m = (M + 2 * BM_CTA - 1) / (2 * BM_CTA);
+    const long t256 = tiles_m * ((N + 255) / 256), t128 = tiles_m * ((N + 127) / 128);
+    const long r256 = (t256 + pairs_avail - 1) / pairs_avail, r128 = (t128 + pairs_avail - 1) / pairs_avail;
+    const bool narrow = 0.87 * (double)r128 < (double)r256 - 1e-9;
+    *tiles = narrow ? t128 : t256;
+    return narrow;
+}
+
+bool tc_shape_ok(const lrq_layer* L) {
+    // shapes this kernel takes: whole 64-wide k-blocks that never straddle a TLQ group; 16-byte aligned code rows
+    if (L->K % BK || L->group % BK) return false;
+    if (L->w_bits < 3 || L->w_bits > 4) return false;       // 2-bit tables take the CUDA-core kernel
+    if (L->packed3) return false;                            // true 3-bit packing takes the small-M kernel
+    return lrq_aligned(L->levels, 16) && lrq_aligned(L->codes, 16);
+}
+
+bool make_w_map(const lrq_layer* L, bool narrow, CUtensorMap* tm) {
+    const uint64_t w_row = (uint64_t)L->K / 2;
+    return lrq_tma::make_map_2d(tm, L->codes, 1, (uint64_t)L->N, w_row, w_row, BK / 2, narrow ? 64 : 128, false);
+}
+
 }  // namespace
+
+void lrq_qgemm_tc_prepare(lrq_layer* L) {
+    L->have_tm_w = tc_shape_ok(L) && make_w_map(L, false, &L->tm_w_wide) && make_w_map(L, true, &L->tm_w_narrow);
+}
 
 lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                                const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st) {
-    // shapes this kernel takes: whole 64-wide k-blocks that never straddle a TLQ group; 16-byte aligned code rows
-    if (L->K % BK || L->group % BK) return LRQ_ERR_UNSUPPORTED;
-    if (L->w_bits < 3 || L->w_bits > 4) return LRQ_ERR_UNSUPPORTED;   // 2-bit tables take the CUDA-core kernel
-    if (!lrq_aligned(L->levels, 16) || !lrq_aligned(L->codes, 16) || !lrq_aligned(a_codes, 16)) return LRQ_ERR_UNSUPPORTED;
+    if (!tc_shape_ok(L) || !lrq_aligned(a_codes, 16)) return LRQ_ERR_UNSUPPORTED;
     const size_t es = dt == LRQ_F32 ? 4 : 2;
     if (!lrq_aligned(Y, 16) || ((size_t)ldy * es) % 16) return LRQ_ERR_UNSUPPORTED;
     const int ab = L->act.a_bits;
@@ -652,28 +692,24 @@ lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const
     p.levels = L->levels; p.wsum = L->wsum; p.wscale = L->wscale; p.bias = L->bias;
     p.Y = Y; p.ldy = ldy; p.M = M; p.N = L->N; p.K = L->K; p.G = L->group; p.y_dtype = (int)dt;
     p.status = lrq_status_word();
-    // code matrices as byte tensors: a tile is 128 rows by one k-block of codes
-    const uint64_t a_row = (uint64_t)L->K * ab / 8, w_row = (uint64_t)L->K / 2;
-    // Tile width.  A 128-wide tile was measured at about 0.87 of the time of a 256-wide one (the weight decode
-    // halves; the activation expansion, the hand-overs and the epilogue set-up do not), so it only pays when it
-    // cuts the number of rounds of tiles over the CTA pairs: small M with a narrow or ragged N (80 wide tiles on
-    // 74 pairs are two rounds, the same work as 144 narrow tiles is two cheaper rounds).
-    int dev = 0, sms = 0;
-    LRQ_CUDA_TRY(cudaGetDevice(&dev));
-    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const long pairs_avail = sms / 2 > 0 ? sms / 2 : 1;
-    const long tiles_m = (M + 2 * BM_CTA - 1) / (2 * BM_CTA);
-    const long t256 = tiles_m * ((L->N + 255) / 256), t128 = tiles_m * ((L->N + 127) / 128);
-    const long r256 = (t256 + pairs_avail - 1) / pairs_avail, r128 = (t128 + pairs_avail - 1) / pairs_avail;
-    const bool narrow = 0.87 * (double)r128 < (double)r256 - 1e-9;
-    CUtensorMap tmA, tmW;
+    int sms = 0;
+    if (lrq_current_device(nullptr, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
+    long tiles = 0;
+    const bool narrow = narrow_tiles(M, L->N, sms, &tiles);
+    // code matrices as byte tensors: a tile is 128 rows by one k-block of codes.  The weight side comes from the
+    // layer handle; the activation codes and the output depend on this call's pointers and M.
+    const uint64_t a_row = (uint64_t)L->K * ab / 8;
+    CUtensorMap tmA, tmW_local;
+    const CUtensorMap* tmW = narrow ? &L->tm_w_narrow : &L->tm_w_wide;
+    if (!L->have_tm_w) {
+        if (!make_w_map(L, narrow, &tmW_local)) return LRQ_ERR_CUDA;
+        tmW = &tmW_local;
+    }
     if (!lrq_tma::make_map_2d(&tmA, a_codes, 1, (uint64_t)M, a_row, a_row, BK * ab / 8, BM_CTA, false)) return LRQ_ERR_CUDA;
-    if (!lrq_tma::make_map_2d(&tmW, L->codes, 1, (uint64_t)L->N, w_row, w_row, BK / 2, narrow ? 64 : 128, false)) return LRQ_ERR_CUDA;
     // outputs leave through TMA stores of 32-row tiles, 128 bytes wide (32 fp32 or 64 16-bit columns)
     CUtensorMap tmY;
     if (!lrq_tma::make_map_2d(&tmY, Y, (int)es, (uint64_t)M, (uint64_t)L->N, (uint64_t)ldy, dt == LRQ_F32 ? 32 : 64, 32, true)) return LRQ_ERR_CUDA;
-    const int tiles = (int)(narrow ? t128 : t256);
-#define LRQ_GO(AB, WB) return narrow ? launch<AB, WB, 128>(p, tmA, tmW, tmY, tiles, st) : launch<AB, WB, 256>(p, tmA, tmW, tmY, tiles, st)
+#define LRQ_GO(AB, WB) return narrow ? launch<AB, WB, 128>(p, tmA, *tmW, tmY, (int)tiles, st) : launch<AB, WB, 256>(p, tmA, *tmW, tmY, (int)tiles, st)
     if (ab == 8 && L->w_bits == 4) LRQ_GO(8, 4);
     if (ab == 8) LRQ_GO(8, 3);
     if (ab == 4 && L->w_bits == 4) LRQ_GO(4, 4);

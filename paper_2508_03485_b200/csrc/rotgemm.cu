@@ -14,6 +14,7 @@
 #include "lrq_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tma_host.cuh"
+#include <mutex>
 
 namespace {
 using namespace lrq_tc;
@@ -69,6 +70,8 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    lrq_pdl_trigger();
+    lrq_pdl_wait();                      // the set-up above overlaps the previous kernel's tail; X may be its output
 
     if (warp == PRODUCER_WARP) {
         if (lane == 0) {
@@ -205,85 +208,33 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     }
 }
 
-// ---- plain CUDA-core kernel for shapes the tensor-core kernel does not take ---------------------------
-constexpr int TM = 64, TN = 64, TK = 32;
-
-__global__ void __launch_bounds__(256)
-rotgemm_simple_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx,
-                      const __nv_bfloat16* __restrict__ R, float* __restrict__ Y) {
-    __shared__ float Xs[TK][TM + 1];
-    __shared__ float Rs[TK][TN + 1];
-    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
-    float acc[4][4] = {};
-    for (int k0 = 0; k0 < K; k0 += TK) {
-        for (int e = tid; e < TM * TK; e += 256) {
-            const int r = e / TK, kk = e % TK, m = m0 + r, k = k0 + kk;
-            Xs[kk][r] = (m < M && k < K) ? __bfloat162float(X[(size_t)m * ldx + k]) : 0.f;
-        }
-        for (int e = tid; e < TN * TK; e += 256) {
-            const int kk = e / TN, c = e % TN, k = k0 + kk, n = n0 + c;
-            Rs[kk][c] = (k < K && n < K) ? __bfloat162float(R[(size_t)k * K + n]) : 0.f;
-        }
-        __syncthreads();
-#pragma unroll 8
-        for (int kk = 0; kk < TK; ++kk) {
-            float a[4], b[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { a[i] = Xs[kk][ty * 4 + i]; b[i] = Rs[kk][tx * 4 + i]; }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int m = m0 + ty * 4 + i;
-        if (m >= M) continue;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int n = n0 + tx * 4 + j;
-            if (n < K) Y[(size_t)m * K + n] = acc[i][j];
-        }
-    }
-}
-
 }  // namespace
 
 lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y,
-                              int* ext_min, int* ext_max, bool* have_ext, cudaStream_t st) {
-    if (have_ext) *have_ext = false;
-    // TMA needs 16-byte aligned bases and row pitches; the fp32 rows are stored with 128-bit stores
-    const bool tc_ok = (K % 8) == 0 && (ldx % 8) == 0 && lrq_aligned(X, 16) && lrq_aligned(R, 16) && lrq_aligned(Y, 16);
-    if (tc_ok) {
-        CUtensorMap tmX, tmR;
-        if (!lrq_tma::make_map_2d(&tmX, X, 2, (uint64_t)M, (uint64_t)K, (uint64_t)ldx, BK, BM, true)) return LRQ_ERR_CUDA;
-        if (!lrq_tma::make_map_2d(&tmR, R, 2, (uint64_t)K, (uint64_t)K, (uint64_t)K, 64, BK, true)) return LRQ_ERR_CUDA;
-        static bool configured = false;
-        if (!configured) {
+                              int* ext_min, int* ext_max, cudaStream_t st) {
+    // TMA needs 16-byte aligned bases and row pitches (K and ldx multiples of 8 elements); the C ABI has already
+    // refused anything else
+    if ((K % 8) || (ldx % 8) || !lrq_aligned(X, 16) || !lrq_aligned(R, 16) || !lrq_aligned(Y, 16) || !ext_min || !ext_max)
+        return LRQ_ERR_INVALID_ARG;
+    CUtensorMap tmX, tmR;
+    if (!lrq_tma::make_map_2d(&tmX, X, 2, (uint64_t)M, (uint64_t)K, (uint64_t)ldx, BK, BM, true)) return LRQ_ERR_CUDA;
+    if (!lrq_tma::make_map_2d(&tmR, R, 2, (uint64_t)K, (uint64_t)K, (uint64_t)K, 64, BK, true)) return LRQ_ERR_CUDA;
+    int dev = 0, sms = 0;
+    if (lrq_current_device(&dev, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
+    {   // the shared-memory opt-in is a per-device function attribute: set once per device
+        static std::mutex mu;
+        static bool configured[LRQ_MAX_DEVICES] = {};
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[dev]) {
             LRQ_CUDA_TRY(cudaFuncSetAttribute(rotgemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-            configured = true;
+            configured[dev] = true;
         }
-        int dev = 0, sms = 0;
-        LRQ_CUDA_TRY(cudaGetDevice(&dev));
-        LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        const int tiles = ((M + BM - 1) / BM) * ((K + BN - 1) / BN);
-        const bool ext = ext_min && ext_max;
-        if (ext) {          // identity elements of the integer min / max: bytes 0x7f.. (a huge float), 0x80.. (a hugely negative one)
-            LRQ_CUDA_TRY(cudaMemsetAsync(ext_min, 0x7f, (size_t)M * sizeof(int), st));
-            LRQ_CUDA_TRY(cudaMemsetAsync(ext_max, 0x80, (size_t)M * sizeof(int), st));
-        }
-        rotgemm_tc_kernel<<<tiles < sms ? tiles : sms, NUM_THREADS, SMEM_BYTES, st>>>(tmX, tmR, Y, M, K, ext ? ext_min : nullptr,
-                                                                                    ext ? ext_max : nullptr, lrq_status_word());
-        if (have_ext) *have_ext = ext;
-        LRQ_CUDA_TRY(cudaGetLastError());
-        return LRQ_OK;
     }
-    dim3 grid((K + TN - 1) / TN, (M + TM - 1) / TM), block(256);
-    rotgemm_simple_kernel<<<grid, block, 0, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx,
-                                                  static_cast<const __nv_bfloat16*>(R), Y);
-    LRQ_CUDA_TRY(cudaGetLastError());
+    const int tiles = ((M + BM - 1) / BM) * ((K + BN - 1) / BN);
+    // identity elements of the integer min / max: bytes 0x7f.. (a huge float), 0x80.. (a hugely negative one)
+    LRQ_CUDA_TRY(cudaMemsetAsync(ext_min, 0x7f, (size_t)M * sizeof(int), st));
+    LRQ_CUDA_TRY(cudaMemsetAsync(ext_max, 0x80, (size_t)M * sizeof(int), st));
+    LRQ_CUDA_TRY(lrq_launch_pdl(rotgemm_tc_kernel, dim3(tiles < sms ? tiles : sms), dim3(NUM_THREADS), SMEM_BYTES, st, tmX, tmR,
+                                Y, M, K, ext_min, ext_max, lrq_status_word()));
     return LRQ_OK;
 }

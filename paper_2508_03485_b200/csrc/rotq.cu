@@ -6,9 +6,14 @@
 // memory.  The 1/sqrt(B) normalisation is never applied to the elements: it is folded into the
 // per-token scale, since rint(y/s) is invariant under a common factor of y and s.
 #include "lrq_internal.cuh"
+#include "f32x2.cuh"
+#include "rotq_common.cuh"
 #include <climits>
+#include <mutex>
+#include <vector>
 
 namespace {
+using namespace lrq_rq;
 
 __device__ __forceinline__ void bfly8(float* v) {
 #pragma unroll
@@ -26,10 +31,6 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& r, float* v) {
         v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
     }
 }
-
-// Per-token quantization parameters from the token's extremes of the un-normalised transform.
-// s_u is the step in the un-normalised domain; the reported scale is s_u * nrm.
-struct TokenQ { float inv; float negz; };
 
 __device__ __forceinline__ TokenQ token_params(float mn, float mx, float amax, int a_bits, int mode, double nrm,
                                                float* scale_out, int32_t* zp_out) {
@@ -60,9 +61,7 @@ __device__ __forceinline__ int quant1(float u, const TokenQ& t, int qmax) {
 // ------------------------------------------------------------------------------------------------
 // Generic kernel: one CTA per token, the token's K transformed values live in shared memory.
 // Any B = 2^n (8..4096) dividing K, any K that is a multiple of 8.
-// SRC_F32: the input is an fp32 matrix that is already rotated (dense path): no transform.
 // ------------------------------------------------------------------------------------------------
-template <bool SRC_F32>
 __global__ void __launch_bounds__(256)
 rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log2B, int a_bits, int mode,
                     const float* __restrict__ prescale,
@@ -73,11 +72,10 @@ rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log
     const int m = blockIdx.x;
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int nchunk = K >> 3;
+    lrq_pdl_trigger();
+    lrq_pdl_wait();
 
-    if (SRC_F32) {
-        const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(Xv) + (size_t)m * ldx);
-        for (int c = tid; c < (K >> 2); c += nthr) reinterpret_cast<float4*>(row)[c] = src[c];
-    } else {
+    {
         const uint4* src = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(Xv) + (size_t)m * ldx);
         for (int c = tid; c < nchunk; c += nthr) {
             float v[8];
@@ -92,29 +90,27 @@ rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log
         }
     }
     __syncthreads();
-    if (!SRC_F32) {
-        // remaining stages, up to three index bits per pass
-        for (int bit = 3; bit < log2B; bit += 3) {
-            const int nb = min(3, log2B - bit);           // bits handled in this pass
-            const int span = 1 << nb;
-            const int ngroups = K >> nb;
-            const int lowmask = (1 << bit) - 1;
-            for (int g = tid; g < ngroups; g += nthr) {
-                // g enumerates indices with the nb bits [bit, bit+nb) removed
-                const int base = ((g & ~lowmask) << nb) | (g & lowmask);
-                float v[8];
+    // remaining stages, up to three index bits per pass
+    for (int bit = 3; bit < log2B; bit += 3) {
+        const int nb = min(3, log2B - bit);           // bits handled in this pass
+        const int span = 1 << nb;
+        const int ngroups = K >> nb;
+        const int lowmask = (1 << bit) - 1;
+        for (int g = tid; g < ngroups; g += nthr) {
+            // g enumerates indices with the nb bits [bit, bit+nb) removed
+            const int base = ((g & ~lowmask) << nb) | (g & lowmask);
+            float v[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = (i < span) ? row[base + (i << bit)] : 0.f;
-                if (nb == 3) bfly8(v);
-                else if (nb == 2) {
-                    float a = v[0] + v[1], b = v[0] - v[1], c = v[2] + v[3], d = v[2] - v[3];
-                    v[0] = a + c; v[1] = b + d; v[2] = a - c; v[3] = b - d;
-                } else { float a = v[0], b = v[1]; v[0] = a + b; v[1] = a - b; }
+            for (int i = 0; i < 8; ++i) v[i] = (i < span) ? row[base + (i << bit)] : 0.f;
+            if (nb == 3) bfly8(v);
+            else if (nb == 2) {
+                float a = v[0] + v[1], b = v[0] - v[1], c = v[2] + v[3], d = v[2] - v[3];
+                v[0] = a + c; v[1] = b + d; v[2] = a - c; v[3] = b - d;
+            } else { float a = v[0], b = v[1]; v[0] = a + b; v[1] = a - b; }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) if (i < span) row[base + (i << bit)] = v[i];
-            }
-            __syncthreads();
+            for (int i = 0; i < 8; ++i) if (i < span) row[base + (i << bit)] = v[i];
         }
+        __syncthreads();
     }
     // token extremes
     float mn = INFINITY, mx = -INFINITY, am = 0.f;
@@ -129,7 +125,7 @@ rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log
     __syncthreads();
     if (tid == 0) {
         for (int w = 1; w < (nthr >> 5); ++w) { mn = fminf(mn, red_mn[w]); mx = fmaxf(mx, red_mx[w]); am = fmaxf(am, red_am[w]); }
-        const double nrm = SRC_F32 ? 1.0 : 1.0 / sqrt((double)(1 << log2B));
+        const double nrm = 1.0 / sqrt((double)(1 << log2B));
         tq = token_params(mn, mx, am, a_bits, mode, nrm, scale + m, zp + m);
     }
     __syncthreads();
@@ -168,16 +164,7 @@ rotq_generic_kernel(const void* __restrict__ Xv, int M, int K, long ldx, int log
 // codes) per thread, contiguous across the warp.
 // ------------------------------------------------------------------------------------------------
 constexpr int EPT = 32;
-typedef unsigned long long f32x2;      // two fp32 values in one 64-bit register pair
-
-__device__ __forceinline__ f32x2 pack2(float a, float b) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
-__device__ __forceinline__ void unpack2(f32x2 r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
-__device__ __forceinline__ float min3(float a, float b, float c) { float d; asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
-__device__ __forceinline__ float max3(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
+using namespace lrq_f2;
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
     uint4 r;
@@ -203,52 +190,6 @@ __device__ __forceinline__ void load_raw(const __nv_bfloat16* p, uint4* raw) {
     }
 }
 
-__device__ __forceinline__ uint32_t pack_u8x4(int q0, int q1, int q2, int q3) {
-    uint32_t t, d;
-    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(q3), "r"(q2), "r"(0));
-    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(q1), "r"(q0), "r"(t));
-    return d;
-}
-
-__device__ __forceinline__ uint32_t pack_u4x8(const int* q) {
-    uint32_t t = 0;
-#pragma unroll
-    for (int i = 3; i >= 0; --i)
-        asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(q[2 * i + 1]), "r"(q[2 * i]), "r"(t));
-    return t;
-}
-
-// The same parameters for the fast kernel, where every warp works them out: one fp64 reciprocal refined
-// from the fp32 approximation (two Newton steps, relative error below 1e-14) instead of fp64 divisions.
-__device__ __forceinline__ TokenQ token_params_fast(float mn, float mx, int a_bits, int mode, double nrm,
-                                                    float* scale_out, int32_t* zp_out) {
-    const bool asym = mode == LRQ_ACT_ASYM;
-    const double qsteps = asym ? (double)((1 << a_bits) - 1) : (double)((1 << (a_bits - 1)) - 1);
-    const double range = asym ? (double)mx - (double)mn : (double)fmaxf(fabsf(mn), fabsf(mx));
-    const float r0 = __frcp_rn((float)range);
-    double s, inv;
-    if (range > 0.0 && r0 > 0.f && r0 < 3.0e38f) {
-        double r = (double)r0;
-        r = fma(r, fma(-range, r, 1.0), r);
-        r = fma(r, fma(-range, r, 1.0), r);
-        inv = qsteps * r;
-        s = range * (1.0 / qsteps);
-    } else if (range > 0.0) {      // outside fp32's reciprocal range: plain division
-        s = range / qsteps;
-        inv = 1.0 / s;
-    } else {                       // empty range: unit step in the normalised domain
-        s = 1.0 / nrm;
-        inv = nrm;
-    }
-    const double z = asym ? rint((double)mn * inv) : -(double)(1 << (a_bits - 1));
-    *scale_out = (float)(s * nrm);
-    *zp_out = (int32_t)z;
-    TokenQ t;
-    t.inv = (float)inv;
-    t.negz = (float)(-z);
-    return t;
-}
-
 template <int LOG2B, int A_BITS, int MAX_THREADS, int MIN_CTAS, bool WIDE>
 __global__ void __launch_bounds__(MAX_THREADS, MIN_CTAS)
 rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, int mode, int tok_per_cta, int num_groups,
@@ -266,6 +207,8 @@ rotq_fast_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, in
     const bool seg_leader = lane == seg_lane;
     for (int i = tid; i < 3 * 2 * tok_per_cta; i += blockDim.x) ext[i] = (i & 1) ? INT_MIN : INT_MAX;
     __syncthreads();
+    lrq_pdl_trigger();
+    lrq_pdl_wait();                      // X may be the previous kernel's output; the code buffer may still be read by it
 
     uint4 raw[4];
     {
@@ -445,6 +388,8 @@ rotq_big_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, long ldx, int
     const bool seg_leader = lane == seg_lane;
     for (int i = tid; i < 3 * 2 * tok_per_cta; i += blockDim.x) ext[i] = (i & 1) ? INT_MIN : INT_MAX;
     __syncthreads();
+    lrq_pdl_trigger();
+    lrq_pdl_wait();                      // X may be the previous kernel's output; the code buffer may still be read by it
 
     uint4 raw[4];
     {
@@ -596,6 +541,8 @@ quant_rows_f32_kernel(const float* __restrict__ Y, int M, int K, int mode, uint8
                       float* scale, int32_t* zp) {
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
+    lrq_pdl_trigger();
+    lrq_pdl_wait();                      // the rows and their extremes are the rotation kernel's output
     for (int m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; m < M; m += warps) {
         TokenQ t;
         t.inv = 0.f; t.negz = 0.f;
@@ -635,14 +582,12 @@ quant_rows_f32_kernel(const float* __restrict__ Y, int M, int K, int mode, uint8
 lrq_status lrq_launch_quantize_f32_ext(const float* Y, int M, int K, int a_bits, int mode, uint8_t* codes,
                                        float* scale, int32_t* zp, cudaStream_t st) {
     if (!lrq_aligned(Y, 32)) return LRQ_ERR_INVALID_ARG;          // rows are K*4 bytes with K % 8 == 0: 32-byte aligned chunks
-    int dev = 0, sms = 0;
-    LRQ_CUDA_TRY(cudaGetDevice(&dev));
-    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    int sms = 0;
+    if (lrq_current_device(nullptr, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
     const int blocks_needed = (M + 7) / 8;                        // 8 warps per CTA, one token per warp and step
     const int grid = blocks_needed < sms * 8 ? blocks_needed : sms * 8;
-    if (a_bits == 8) quant_rows_f32_kernel<8><<<grid, 256, 0, st>>>(Y, M, K, mode, codes, scale, zp);
-    else quant_rows_f32_kernel<4><<<grid, 256, 0, st>>>(Y, M, K, mode, codes, scale, zp);
-    LRQ_CUDA_TRY(cudaGetLastError());
+    if (a_bits == 8) LRQ_CUDA_TRY(lrq_launch_pdl(quant_rows_f32_kernel<8>, dim3(grid), dim3(256), 0, st, Y, M, K, mode, codes, scale, zp));
+    else LRQ_CUDA_TRY(lrq_launch_pdl(quant_rows_f32_kernel<4>, dim3(grid), dim3(256), 0, st, Y, M, K, mode, codes, scale, zp));
     return LRQ_OK;
 }
 
@@ -709,9 +654,8 @@ __global__ void ars_finish_kernel(const double* __restrict__ acc, double count, 
 
 lrq_status lrq_launch_ars_metric(const void* X, int M, int K, long ldx, double thr, float* J, int* kind, double* acc,
                                  cudaStream_t st) {
-    int dev = 0, sms = 0;
-    LRQ_CUDA_TRY(cudaGetDevice(&dev));
-    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    int sms = 0;
+    if (lrq_current_device(nullptr, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
     LRQ_CUDA_TRY(cudaMemsetAsync(acc, 0, sizeof(double), st));
     long blocks = ((long)M + 7) / 8;                         // 8 warps per CTA, one row per warp and step
     if (blocks > (long)sms * 8) blocks = (long)sms * 8;
@@ -722,16 +666,36 @@ lrq_status lrq_launch_ars_metric(const void* X, int M, int K, long ldx, double t
     return LRQ_OK;
 }
 
-static lrq_status launch_generic(bool f32, const void* X, int M, int K, long ldx, int log2B, int a_bits, int mode, const float* prescale,
+// CTAs of `kern` (with this CTA size and dynamic shared memory) that one SM keeps resident.  The answer, and the
+// shared-memory opt-in it needs (a per-device function attribute), are worked out once per (kernel, device, shape)
+// under a lock and remembered: the launch path itself then makes no runtime query.
+static lrq_status resident_ctas(const void* kern, int dev, int threads, size_t smem, int* per_sm) {
+    struct Entry { const void* kern; int dev, threads; size_t smem; int per_sm; };
+    static std::mutex mu;
+    static std::vector<Entry> cache;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Entry& e : cache)
+        if (e.kern == kern && e.dev == dev && e.threads == threads && e.smem == smem) { *per_sm = e.per_sm; return LRQ_OK; }
+    if (smem > 40 * 1024) LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int n = 0;
+    LRQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, threads, smem));
+    if (n < 1) return LRQ_ERR_UNSUPPORTED;
+    cache.push_back({kern, dev, threads, smem, n});
+    *per_sm = n;
+    return LRQ_OK;
+}
+
+static lrq_status launch_generic(const void* X, int M, int K, long ldx, int log2B, int a_bits, int mode, const float* prescale,
                                  uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st) {
     const size_t smem = (size_t)K * sizeof(float);
     if (smem > 200 * 1024) return LRQ_ERR_UNSUPPORTED;
-    auto kern = f32 ? rotq_generic_kernel<true> : rotq_generic_kernel<false>;
-    if (smem > 40 * 1024)
-        LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int dev = 0, per_sm = 0;
+    if (lrq_current_device(&dev, nullptr) != LRQ_OK) return LRQ_ERR_CUDA;
     const int threads = (K >= 2048) ? 256 : (K >= 1024 ? 128 : 64);
-    kern<<<M, threads, smem, st>>>(X, M, K, ldx, log2B, a_bits, mode, prescale, codes, scale, zp);
-    LRQ_CUDA_TRY(cudaGetLastError());
+    lrq_status rs = resident_ctas(reinterpret_cast<const void*>(rotq_generic_kernel), dev, threads, smem, &per_sm);   // sets the shared-memory opt-in
+    if (rs != LRQ_OK) return rs;
+    LRQ_CUDA_TRY(lrq_launch_pdl(rotq_generic_kernel, dim3(M), dim3(threads), smem, st, X, M, K, ldx, log2B, a_bits, mode, prescale, codes,
+                                scale, zp));
     return LRQ_OK;
 }
 
@@ -771,17 +735,15 @@ static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits,
     else if (threads <= 384) kern = LRQ_PICK(384, 2);
     else kern = LRQ_PICK(512, 1);
 #undef LRQ_PICK
-    if (smem > 40 * 1024) LRQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     // persistent grid: as many CTAs as stay resident, each walking over token groups with a grid stride
     int dev = 0, sms = 0, per_sm = 0;
-    LRQ_CUDA_TRY(cudaGetDevice(&dev));
-    LRQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    LRQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem));
-    if (per_sm < 1) return LRQ_ERR_UNSUPPORTED;
+    if (lrq_current_device(&dev, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
+    lrq_status rs = resident_ctas(reinterpret_cast<const void*>(kern), dev, threads, smem, &per_sm);
+    if (rs != LRQ_OK) return rs;
     const int groups = (M + T - 1) / T;
     const int grid = groups < sms * per_sm ? groups : sms * per_sm;
-    kern<<<grid, threads, smem, st>>>(static_cast<const __nv_bfloat16*>(X), M, K, ldx, mode, T, groups, prescale, codes, scale, zp);
-    LRQ_CUDA_TRY(cudaGetLastError());
+    LRQ_CUDA_TRY(lrq_launch_pdl(kern, dim3(grid), dim3(threads), smem, st, static_cast<const __nv_bfloat16*>(X), M, K, ldx, mode, T,
+                                groups, prescale, codes, scale, zp));
     return LRQ_OK;
 }
 
@@ -804,10 +766,5 @@ lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B
         }
         if (r != LRQ_ERR_UNSUPPORTED) return r;
     }
-    return launch_generic(false, X, M, K, ldx, log2B, a_bits, mode, prescale, codes, scale, zp, st);
-}
-
-lrq_status lrq_launch_quantize_f32(const float* Y, int M, int K, long ldy, int a_bits, int mode,
-                                   uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st) {
-    return launch_generic(true, Y, M, K, ldy, 0, a_bits, mode, nullptr, codes, scale, zp, st);
+    return launch_generic(X, M, K, ldx, log2B, a_bits, mode, prescale, codes, scale, zp, st);
 }

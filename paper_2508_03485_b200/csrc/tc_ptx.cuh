@@ -6,8 +6,8 @@
 
 namespace lrq_tc {
 
-// A wait gives up after this many SM clock cycles (a second or two); the kernel then records a code and
-// unwinds.  kWaitLimit bounds the polls of the drain loops that run after such an abort.
+// A wait gives up after `limit` SM clock cycles (default kWaitCycles: a second or two); the kernel then records
+// a code and unwinds.  kWaitLimit bounds the polls of the drain loops that run after such an abort.
 constexpr long long kWaitCycles = 3000000000ll;
 constexpr uint32_t kWaitLimit = 1u << 22;
 // Each poll lets the hardware suspend the thread for up to this many nanoseconds while the phase is
@@ -69,14 +69,15 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 // thread sleeps SLEEP_NS nanoseconds: a warp that spins on try_wait competes for issue slots with the
 // warps that do the work, and most waiters here (epilogue, TMA producer) are far from the critical path.
 template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                          long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     do {
         if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-    } while (clock64() - t0 < kWaitCycles);
+    } while (clock64() - t0 < limit);
     *abort_flag = 1;
     if (status) atomicCAS(status, 0, code);
     return false;
@@ -85,19 +86,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // observed the phase has no ordering against the asynchronous writes it guards), then the lanes agree
 // on one answer, so that warp-level synchronisation after the wait stays convergent when a wait expires.
 template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
-    const bool ok = mbar_wait<SLEEP_NS>(bar, parity, abort_flag, status, code);
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                               long long limit = kWaitCycles) {
+    const bool ok = mbar_wait<SLEEP_NS>(bar, parity, abort_flag, status, code, limit);
     return __all_sync(0xffffffffu, ok);
 }
 template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                                  long long limit = kWaitCycles) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     const long long t0 = clock64();
     do {
         if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
         if (mbar_try_wait_cluster(bar, parity)) return true;
         if (*abort_flag) return false;
-    } while (clock64() - t0 < kWaitCycles);
+    } while (clock64() - t0 < limit);
     *abort_flag = 1;
     if (status) atomicCAS(status, 0, code);
     return false;

@@ -48,15 +48,15 @@ def test_argument_checks_run_before_any_launch(lib):
     assert lib.lrq_act_workspace_bytes(5, 128, C.byref(p4)) == 2560
     assert lib.lrq_act_workspace_bytes(5, 128, C.byref(p)) == 0
     a = (C.c_double * 1)(1.0)
-    t = _TlqParams(5, 0, 7, 1, 1, a, a)
+    t = _TlqParams(5, 0, 7, 1, 1, a, a, 0)
     assert lib.lrq_tlq_quantize_weights(fake, 8, 64, C.byref(t), fake, fake, None, fake, None, 0, None) == 2
-    t = _TlqParams(4, 48, 7, 1, 1, a, a)    # group does not divide K
+    t = _TlqParams(4, 48, 7, 1, 1, a, a, 0)    # group does not divide K
     assert lib.lrq_tlq_quantize_weights(fake, 8, 64, C.byref(t), fake, fake, None, fake, None, 0, None) == 2
     h = C.c_void_p()
-    assert lib.lrq_layer_create(C.byref(h), 8, 64, 4, 0, None, fake, fake, None, None, C.byref(p)) == 1
-    assert lib.lrq_layer_create(C.byref(h), 8, 64, 4, 0, fake, fake, fake, None, None, C.byref(p)) == 2  # 128 does not divide 64
+    assert lib.lrq_layer_create(C.byref(h), 8, 64, 4, 0, 0, None, fake, fake, None, None, C.byref(p)) == 1
+    assert lib.lrq_layer_create(C.byref(h), 8, 64, 4, 0, 0, fake, fake, fake, None, None, C.byref(p)) == 2  # 128 does not divide 64
     p5 = _ActParams(1, 64, None, 8, 0)
-    assert lib.lrq_layer_create(C.byref(h), 8, 64, 4, 0, fake, fake, fake, None, None, C.byref(p5)) == 0
+    assert lib.lrq_layer_create(C.byref(h), 8, 64, 4, 0, 0, fake, fake, fake, None, None, C.byref(p5)) == 0
     assert lib.lrq_workspace_bytes(h, 10) == 768 + 256 + 256
     assert lib.lrq_qlinear(h, fake, 10, 64, fake, 0, 8, None, 0, None) == 3       # workspace missing
     assert lib.lrq_qlinear(h, fake, 10, 64, fake, 0, 4, fake, 1 << 20, None) == 1  # ldy < N
