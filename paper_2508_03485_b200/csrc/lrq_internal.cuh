@@ -61,6 +61,9 @@ inline cudaError_t lrq_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block,
 // rotq.cu
 lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B, int a_bits, int mode, const float* prescale,
                                     uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
+// rotq_blk.cu : the same for blocks of 8..128 channels with K a multiple of 128; LRQ_ERR_UNSUPPORTED otherwise
+lrq_status lrq_launch_rotq_blk(const void* X, int M, int K, long ldx, int B, int a_bits, int mode, const float* prescale,
+                               uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st);
 // rotgemm.cu : Y[M,K] (fp32) = X[M,K] (bf16) . R[K,K] (bf16) on the tensor cores; also leaves every row's minimum and
 // maximum in ext_min[M] / ext_max[M] as order-preserving integers.
 lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y,

@@ -749,6 +749,11 @@ static lrq_status launch_fast(const void* X, int M, int K, long ldx, int a_bits,
 
 lrq_status lrq_launch_rotq_hadamard(const void* X, int M, int K, long ldx, int B, int a_bits, int mode, const float* prescale,
                                     uint8_t* codes, float* scale, int32_t* zp, cudaStream_t st) {
+    // blocks of up to 128 channels: whole blocks per thread, TMA-fed (rotq_blk.cu), when the shape allows
+    {
+        const lrq_status r = lrq_launch_rotq_blk(X, M, K, ldx, B, a_bits, mode, prescale, codes, scale, zp, st);
+        if (r != LRQ_ERR_UNSUPPORTED) return r;
+    }
     int log2B = 0;
     while ((1 << log2B) < B) ++log2B;
     // the fast kernel needs whole 32-element thread slices and, for B >= 2048, whole-CTA tokens

@@ -41,4 +41,18 @@ inline bool make_map_2d(CUtensorMap* tm, const void* ptr, int elem_bytes, uint64
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row-major bf16 matrix [rows, cols] (cols a multiple of 64, `ld` elements between rows) seen as a 3-D tensor
+// [rows][cols / 64][64], so that one copy brings `box_rows` whole rows into shared memory as consecutive 128-byte
+// lines (64 elements each), 128-byte swizzled: the 16-byte chunk c of line L lands at chunk c ^ (L & 7).
+inline bool make_map_rows_bf16(CUtensorMap* tm, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc || cols % 64 || cols / 64 > 256 || box_rows < 1 || box_rows > 256) return false;
+    const cuuint64_t dims[3] = {64, cols / 64, rows};
+    const cuuint64_t strides[2] = {128, ld * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)(cols / 64), box_rows};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace lrq_tma
