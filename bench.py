@@ -201,7 +201,10 @@ class Workload:
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            tl = P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid)
+            # 3-bit codes of a small batch are stored in their true packing (eight codes in three bytes): such a layer
+            # is bound by streaming its weights once, and the small-tile contraction reads that layout
+            layout = P.CODES_PACKED3 if (s.w_bits == 3 and s.M <= 512) else P.CODES_NIBBLE
+            tl = P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid, code_layout=layout)
             e1.record()
             torch.cuda.synchronize()
             self.tlq_ms += e0.elapsed_time(e1)
@@ -279,13 +282,32 @@ def kernel_objects(P, torch, W, timed, peaks, out_name, gemm_impl=0, want_dense=
     big = max(range(len(specs)), key=lambda i: specs[i].N * specs[i].K * specs[i].M)
     s, L = specs[big], layers[big]
     q, sc, zp = P.lrq_rotate_quantize_act(W.Xs[big], L.kind, s.a_bits, s.had_block, L.R)
-    gemm_ms = float(np.mean(timed(lambda: P.lrq_qgemm_codes(L, q, sc, zp, W.ydt, gemm_impl, W.Ys[big], stream), 20)))
+    impl = 2 if L.tlq.code_layout == P.CODES_PACKED3 else gemm_impl
+    gq = torch.cuda.CUDAGraph()                       # one launch per replay: no host call inside the timed events
+    P.lrq_qgemm_codes(L, q, sc, zp, W.ydt, impl, W.Ys[big], stream)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(gq):
+        P.lrq_qgemm_codes(L, q, sc, zp, W.ydt, impl, W.Ys[big])
+    gemm_ms = float(np.mean(timed(gq.replay, 20)))
     gemm_tf = 2.0 * s.M * s.N * s.K / (gemm_ms * 1e-3) / 1e12
-    out["roofline"] = {"kernel": f"qgemm cfg{cfg} {s.name} {s.M}x{s.N}x{s.K} W{s.w_bits}A{s.a_bits} out {out_name}", "bound": "tensor",
-                       "achieved": gemm_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": gemm_tf / peaks["bf16_tflops"],
-                       "traffic": NCU_TRAFFIC_BYTES.get(f"qgemm cfg{cfg} {s.name}") if out_name == "f32" else None,
-                       "traffic_unit": "bytes per launch (ncu dram read + write)", "algorithmic_flops": 2.0 * s.M * s.N * s.K,
-                       "peak_source": peaks["source"] + " burst bf16 (kernel timed alone)", "ms": gemm_ms}
+    if L.tlq.code_layout == P.CODES_PACKED3:
+        # a small batch: every byte is moved once and the tensor cores idle; algorithmic bytes = activation codes +
+        # 3-bit weight codes + level tables + per-token / per-channel terms + outputs
+        G = s.group if s.group > 0 else s.K
+        esz = 4 if out_name == "f32" else 2
+        nbytes = s.M * s.K * s.a_bits / 8.0 + s.N * s.K * 3 / 8.0 + s.N * (s.K // G) * 8 * 4.0 + 8.0 * s.M + 4.0 * s.N + s.M * s.N * esz
+        gbs = nbytes / (gemm_ms * 1e-3) / 1e9
+        out["roofline"] = {"kernel": f"qgemm (small-tile, packed 3-bit codes) cfg{cfg} {s.name} {s.M}x{s.N}x{s.K} W3A{s.a_bits} out {out_name}",
+                           "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                           "traffic": None, "algorithmic_bytes": nbytes, "tflops": gemm_tf,
+                           "peak_source": peaks["source"] + " copy bandwidth; a launch of a few microseconds is latency-bound, not bandwidth-bound",
+                           "ms": gemm_ms}
+    else:
+        out["roofline"] = {"kernel": f"qgemm cfg{cfg} {s.name} {s.M}x{s.N}x{s.K} W{s.w_bits}A{s.a_bits} out {out_name}", "bound": "tensor",
+                           "achieved": gemm_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": gemm_tf / peaks["bf16_tflops"],
+                           "traffic": NCU_TRAFFIC_BYTES.get(f"qgemm cfg{cfg} {s.name}") if out_name == "f32" else None,
+                           "traffic_unit": "bytes per launch (ncu dram read + write)", "algorithmic_flops": 2.0 * s.M * s.N * s.K,
+                           "peak_source": peaks["source"] + " burst bf16 (kernel timed alone)", "ms": gemm_ms}
     del q, sc, zp
     had = [i for i in range(len(specs)) if specs[i].rot == "hadamard"]
     if had:
@@ -451,7 +473,7 @@ def run_cuda(args):
                 ent = {"config": c, "workload": workload_name(c), "layers": len(Wc.specs), "ms_per_step": msc,
                        "value": Wc.flops() / (msc * 1e-3) / 1e12, "unit": UNIT,
                        "tokens_per_s": (sum(s_.M for s_ in Wc.specs) / len(Wc.specs)) / (msc * 1e-3)}
-                if c == 3:
+                if c in (3, 0):
                     ent.update(kernel_objects(P, torch, Wc, timed, peaks, args.out_dtype, args.gemm_impl, want_dense=True))
                 per.append(ent)
                 Wc.close(); del Wc
@@ -572,8 +594,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--config", type=int, default=4, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--quick", action="store_true", help="only the chosen workload: no 16-bit-output leg, no per_config list")
-    ap.add_argument("--gemm-impl", type=int, default=0, choices=[0, 1],
-                    help="kernel timed alone for the roofline object: 0 tcgen05, 1 CUDA-core baseline")
+    ap.add_argument("--gemm-impl", type=int, default=0, choices=[0, 1, 2],
+                    help="kernel timed alone for the roofline object: 0 large-tile tcgen05, 1 CUDA-core baseline, 2 small-tile tcgen05")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph replay of the step")
     ap.add_argument("--kernel", default=None, choices=["rotq", "qgemm", "tlq", "ars"], help="time one kernel only")
     ap.add_argument("--layer", type=int, default=0, help="layer index of the workload for --kernel")

@@ -221,8 +221,11 @@ lrq_status lrq_qlinear_stack(const lrq_layer* const* layers, int n_layers,
                              void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Contraction and epilogue alone (Eq. 10), on activation codes produced earlier by
- * lrq_rotate_quantize_act.  `impl`: 0 = tcgen05 tensor-core kernel, 1 = plain CUDA-core kernel
- * (kept as the in-library ablation baseline). No workspace needed. */
+ * lrq_rotate_quantize_act.  `impl`: 0 = large-tile tcgen05 kernel (pairs of CTAs, 256 x 256 tiles), 1 = plain
+ * CUDA-core kernel (kept as the in-library ablation baseline), 2 = small-tile tcgen05 kernel (128 x 32 tiles: the
+ * one lrq_qlinear picks for a few hundred tokens or fewer, and the only tensor-core kernel that reads
+ * LRQ_CODES_PACKED3).  LRQ_ERR_UNSUPPORTED when the kernel asked for does not take the layer's shape.
+ * No workspace needed. */
 lrq_status lrq_qgemm_codes(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                            const int32_t* a_zp, int M, void* Y, lrq_dtype y_dtype, long ldy,
                            int impl, void* cuda_stream);

@@ -98,6 +98,10 @@ lrq_status lrq_launch_qgemm_simple(const lrq_layer* L, const uint8_t* a_codes, c
                                    const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);
 lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                                const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);
+// qgemm_small.cu : 128 x 32 tiles, one CTA each, for small token counts and for packed 3-bit codes
+bool lrq_qgemm_small_takes(const lrq_layer* L);
+lrq_status lrq_launch_qgemm_small(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
+                                  const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);
 // fills the layer's cached TMA descriptors (called once by lrq_layer_create; never fails: without a driver, or for
 // shapes the tensor-core kernel does not take, the layer is simply left without them)
 void lrq_qgemm_tc_prepare(lrq_layer* L);

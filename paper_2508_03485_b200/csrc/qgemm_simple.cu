@@ -18,7 +18,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 cast_out<__nv_bfloat16>(flo
 template <typename OutT>
 __global__ void __launch_bounds__(256)
 qgemm_simple_kernel(const uint8_t* __restrict__ a_codes, const float* __restrict__ a_scale,
-                    const int32_t* __restrict__ a_zp, int M, int N, int K, int a_bits, int w_bits, int G,
+                    const int32_t* __restrict__ a_zp, int M, int N, int K, int a_bits, int w_bits, int G, int packed3,
                     const uint8_t* __restrict__ w_codes, const float* __restrict__ levels,
                     const float* __restrict__ wsum, const float* __restrict__ wscale,
                     const float* __restrict__ bias, OutT* __restrict__ Y, long ldy) {
@@ -44,7 +44,14 @@ qgemm_simple_kernel(const uint8_t* __restrict__ a_codes, const float* __restrict
             const int r = e / TK, kk = e % TK, n = n0 + r, k = k0 + kk;
             float v = 0.f;
             if (n < N && k < K) {
-                const int u = (w_codes[((size_t)n * K + k) >> 1] >> (4 * (k & 1))) & 0xF;
+                int u;
+                if (packed3) {                               // eight codes in three bytes: code j at bits 3j..3j+2
+                    const uint8_t* g = w_codes + (size_t)n * (K / 8 * 3) + (size_t)(k >> 3) * 3;
+                    const uint32_t w24 = (uint32_t)g[0] | ((uint32_t)g[1] << 8) | ((uint32_t)g[2] << 16);
+                    u = (w24 >> (3 * (k & 7))) & 7;
+                } else {
+                    u = (w_codes[((size_t)n * K + k) >> 1] >> (4 * (k & 1))) & 0xF;
+                }
                 v = levels[((size_t)n * ngrp + k / G) * nlev + u];
             }
             Ws[kk][r] = v;
@@ -86,7 +93,7 @@ lrq_status lrq_launch_qgemm_simple(const lrq_layer* L, const uint8_t* a_codes, c
     dim3 grid((L->N + TN - 1) / TN, (M + TM - 1) / TM), block(256);
 #define LRQ_GO(T)                                                                                              \
     qgemm_simple_kernel<T><<<grid, block, 0, st>>>(a_codes, a_scale, a_zp, M, L->N, L->K, L->act.a_bits,       \
-                                                   L->w_bits, L->group, L->codes, L->levels, L->wsum,          \
+                                                   L->w_bits, L->group, L->packed3, L->codes, L->levels, L->wsum, \
                                                    L->wscale, L->bias, static_cast<T*>(Y), ldy)
     if (dt == LRQ_F32) LRQ_GO(float);
     else if (dt == LRQ_F16) LRQ_GO(__half);

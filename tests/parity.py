@@ -233,11 +233,11 @@ def check_tlq(orc, W: np.ndarray, tl, bits: int, group: int, rows=None, what="",
     return T
 
 
-def gpu_layer(spec: LayerSpec, W: np.ndarray, P):
+def gpu_layer(spec: LayerSpec, W: np.ndarray, P, code_layout: int = 0):
     """Quantize weights on the GPU and build the layer handle.  Returns (QLayer, TLQWeights)."""
     g = default_clip_grid()
     Wd = torch.from_numpy(W).cuda()
-    tl = P.lrq_tlq_quantize_weights(Wd, spec.w_bits, spec.group, 7, g, g)
+    tl = P.lrq_tlq_quantize_weights(Wd, spec.w_bits, spec.group, 7, g, g, code_layout=code_layout)
     R = None
     if spec.rot == "dense":
         R = bf16_to_device(spec.rotation_bf16())

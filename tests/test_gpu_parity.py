@@ -119,7 +119,7 @@ def _small_layer(P, orc, M, K, N, w_bits, a_bits, G, B, seed, rot="hadamard"):
     return spec, W, xb, layer, tl, T
 
 
-@pytest.mark.parametrize("impl", [1, 0])
+@pytest.mark.parametrize("impl", [1, 0, 2])
 @pytest.mark.parametrize("M,K,N,w_bits,a_bits,G,B", [
     (70, 256, 72, 4, 8, 0, 128), (129, 1152, 200, 4, 8, 0, 128), (33, 512, 136, 3, 4, 128, 512),
     (256, 1024, 1024, 3, 4, 0, 1024), (5, 128, 8, 4, 4, 64, 64),
@@ -137,8 +137,8 @@ def test_qgemm_from_oracle_codes(P, orc, impl, M, K, N, w_bits, a_bits, G, B):
     try:
         Y = P.lrq_qgemm_codes(layer, qd, sd, zd, P.F32, impl)
     except P.LrqError as e:
-        if impl == 0 and e.code == 2:
-            pytest.skip("shape not taken by the tensor-core kernel")
+        if impl in (0, 2) and e.code == 2:
+            pytest.skip("shape not taken by this tensor-core kernel")
         raise
     assert P.lrq_device_status() == 0
     PU.check_out(Y.cpu().numpy(), Yo, f"qgemm impl{impl}", rel=1e-5, mx=1e-4)
@@ -469,4 +469,62 @@ def test_two_host_threads_on_two_streams(P):
     for outs in results.values():
         for y in outs:
             assert torch.equal(y, ref)
+    assert P.lrq_device_status() == 0
+
+
+# --------------------------------------------------------------- packed 3-bit codes, small-tile contraction
+@pytest.mark.parametrize("M,K,N,a_bits,G,B", [(256, 1024, 1024, 4, 0, 1024), (70, 256, 72, 8, 0, 128), (33, 512, 136, 4, 128, 512),
+                                              (300, 1152, 392, 8, 128, 128), (1, 128, 8, 4, 64, 64)])
+def test_packed3_codes_and_small_tile_kernel(P, orc, M, K, N, a_bits, G, B):
+    # W3 weights stored as the b-bit codes of Eq. 5 really need: eight codes in three bytes.  TLQ must emit the same
+    # codes and tables as for the nibble layout (compared with the oracle bit for bit through the 3-bit unpacking), and
+    # the layer - taken by the small-tile contraction - must reproduce the oracle's outputs element by element.
+    spec = LayerSpec("p3", 33, M, K, N, 3, a_bits, G, "hadamard", B)
+    W, xb = spec.weights(), spec.activations()
+    layer, tl = PU.gpu_layer(spec, W, P, code_layout=P.CODES_PACKED3)
+    assert tl.codes.shape == (N, 3 * K // 8)
+    T = PU.check_tlq(orc, W, tl, 3, G, what="packed3", packed3=True)
+    Yo, oq, os_, oz, Yr = PU.oracle_layer_rows(orc, spec, xb, T)
+    X = PU.bf16_to_device(xb)
+    q, s, z = P.lrq_rotate_quantize_act(X, P.ROT_HADAMARD, a_bits, B)
+    gq, gz = PU.act_codes_to_numpy(q, a_bits), z.cpu().numpy()
+    act = PU.check_act(gq, s.cpu().numpy(), gz, oq, os_, oz, Yr, "hadamard", B, "packed3 codes")
+    for dt in (P.F32, P.F16):
+        Y = P.lrq_qlinear(layer, X, dt)
+        PU.check_layer_out(orc, T, Y.float().cpu().numpy(), gq, gz, Yo, os_, act, "packed3 qlinear")
+    # the same contraction on the CUDA cores reads the packed layout too
+    Yc = P.lrq_qgemm_codes(layer, q, s, z, P.F32, 1)
+    Ys = P.lrq_qgemm_codes(layer, q, s, z, P.F32, 2)
+    rms = Yc.pow(2).mean().sqrt().item()
+    assert ((Ys - Yc).abs().max().item() <= 2e-3 * rms)
+    with pytest.raises(P.LrqError) as e:
+        P.lrq_qgemm_codes(layer, q, s, z, P.F32, 0)          # the large-tile kernel does not read this layout
+    assert e.value.code == 2
+    assert P.lrq_device_status() == 0
+
+
+def test_packed3_needs_three_bit_codes(P):
+    Wd = torch.zeros((8, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(P.LrqError) as e:
+        P.lrq_tlq_quantize_weights(Wd, 4, 0, 7, [1.0], [1.0], code_layout=P.CODES_PACKED3)
+    assert e.value.code == 2
+
+
+@pytest.mark.parametrize("M", [1, 100, 256, 300])
+@pytest.mark.parametrize("w_bits,a_bits", [(4, 8), (3, 4), (4, 4)])
+def test_small_batches_take_the_small_tile_kernel(P, orc, M, w_bits, a_bits):
+    # lrq_qlinear on a few hundred tokens (the automatic choice) against the oracle, nibble layout
+    spec = LayerSpec("sm", 35, M, 512, 264, w_bits, a_bits, 128, "hadamard", 128)
+    W, xb = spec.weights(), spec.activations()
+    layer, tl = PU.gpu_layer(spec, W, P)
+    T = PU.check_tlq(orc, W, tl, w_bits, 128, what="small")
+    Yo, oq, os_, oz, Yr = PU.oracle_layer_rows(orc, spec, xb, T)
+    X = PU.bf16_to_device(xb)
+    q, s, z = P.lrq_rotate_quantize_act(X, P.ROT_HADAMARD, a_bits, 128)
+    gq, gz = PU.act_codes_to_numpy(q, a_bits), z.cpu().numpy()
+    act = PU.check_act(gq, s.cpu().numpy(), gz, oq, os_, oz, Yr, "hadamard", 128, "small codes")
+    Y = P.lrq_qlinear(layer, X, P.F32)
+    PU.check_layer_out(orc, T, Y.cpu().numpy(), gq, gz, Yo, os_, act, "small qlinear")
+    Y2 = P.lrq_qgemm_codes(layer, q, s, z, P.F32, 2)
+    assert torch.equal(Y, Y2)                                # lrq_qlinear took the small-tile kernel
     assert P.lrq_device_status() == 0
