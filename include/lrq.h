@@ -170,15 +170,19 @@ lrq_status lrq_rotate_weights(const float* W, int N, int K, long ldw, const floa
  *   - kind == LRQ_ROT_DENSE needs M*K*4 <= LRQ_STATIC_SCRATCH_BYTES, otherwise the call returns
  *     LRQ_ERR_WORKSPACE and launches nothing (split the tokens into several calls).  The other
  *     kinds use no scratch and have no size limit.
- *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine).  The first
- *     call on each device looks up the device address of the array (a host-side query, no launch);
- *     make that first call before any stream capture.
+ *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine).  Every call
+ *     asks the runtime for the device address of the array (a host-side query, no launch, nothing cached
+ *     here, so a device reset between calls is harmless).  The FIRST call of the process on each device
+ *     may make the runtime load this library's device code, which reserves memory on the driver's side
+ *     and is not allowed while a stream is being captured: make one call (any M, e.g. one token) on each
+ *     device at start-up, before the phase in which allocation is forbidden.
  *   - All calls on a device share the one array.  Its contents after a call are the last rotation's
  *     output; nothing in it has to start at zero, because the rotation overwrites every element the
  *     quantizer reads.  Two calls that may overlap on the GPU (different streams) race on it:
  *     serialise them.
  * ------------------------------------------------------------------------------------------- */
 #define LRQ_STATIC_SCRATCH_BYTES (8u << 20)
+size_t lrq_static_scratch_bytes(void);   /* the value the library was built with */
 
 lrq_status lrq_rotate_quantize_act_static(const void* X_bf16, int M, int K, long ldx, const lrq_act_params* p,
                                           uint8_t* a_codes, float* a_scale, int32_t* a_zp, void* cuda_stream);

@@ -8,5 +8,5 @@ computation.
 from .gen import (  # noqa: F401
     LayerSpec, CONFIGS, config_layers, make_weights, make_activations,
     make_orthogonal, f32_to_bf16_bits, bf16_bits_to_f32, bf16_bits_to_f64,
-    default_clip_grid,
+    default_clip_grid, salient_channels, make_block_rotations, make_staggered_permutation,
 )

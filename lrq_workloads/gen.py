@@ -77,6 +77,44 @@ def make_orthogonal(seed: int, K: int) -> np.ndarray:
     return q
 
 
+def salient_channels(seed: int, K: int, n_salient: int) -> np.ndarray:
+    """The channels make_activations(seed, ., K, n_salient=...) scales up on every token (its first draw)."""
+    rng = np.random.Generator(np.random.PCG64(seed + 1_000_003))
+    return rng.choice(K, size=n_salient, replace=False) if n_salient > 0 else np.zeros(0, dtype=np.int64)
+
+
+def make_block_rotations(seed: int, K: int, Bd: int) -> np.ndarray:
+    """[K/Bd, Bd, Bd] float64: one Haar-distributed orthogonal matrix per block of Bd channels.  Stands in for a
+    block-diagonal outlier-aware rotation, whose construction from calibration data is outside the path."""
+    assert K % Bd == 0
+    rng = np.random.Generator(np.random.PCG64(seed + 3_000_017))
+    out = np.empty((K // Bd, Bd, Bd))
+    for j in range(K // Bd):
+        q, r = np.linalg.qr(rng.standard_normal(size=(Bd, Bd)))
+        out[j] = q * np.sign(np.diag(r))[None, :]
+    return out
+
+
+def make_staggered_permutation(seed: int, K: int, Bd: int, first: np.ndarray | None = None) -> np.ndarray:
+    """int32 [K] index map of a staggered channel reordering: position i of the reordered vector takes channel
+    perm[i].  The channels are put in a ranking (those of ``first`` lead, in the given order; the rest follow in a
+    seeded random order, standing in for a ranking by calibrated range) and dealt over the K/Bd blocks back and
+    forth: ranks 0..nb-1 to blocks 0..nb-1, ranks nb..2nb-1 to blocks nb-1..0, and so on, each pass filling the
+    next slot of every block.  So the leading channels end up spread over different blocks."""
+    assert K % Bd == 0
+    nb = K // Bd
+    rng = np.random.Generator(np.random.PCG64(seed + 4_000_037))
+    first = np.zeros(0, dtype=np.int64) if first is None else np.asarray(first, dtype=np.int64)
+    rest = np.setdiff1d(np.arange(K), first)
+    ranking = np.concatenate([first, rng.permutation(rest)])
+    perm = np.empty(K, dtype=np.int32)
+    for r, ch in enumerate(ranking):
+        p, pos = divmod(r, nb)
+        b = pos if p % 2 == 0 else nb - 1 - pos
+        perm[b * Bd + p] = ch
+    return perm
+
+
 def default_clip_grid() -> np.ndarray:
     """Grid of clipping factors handed to the TLQ search: 1.00, 1.02, ..., 1.60."""
     return np.round(1.0 + 0.02 * np.arange(31), 2)
@@ -93,7 +131,7 @@ class LayerSpec:
     w_bits: int
     a_bits: int
     group: int            # 0 => per output channel
-    rot: str              # "hadamard" | "dense"
+    rot: str              # "hadamard" | "dense" | "dual" (a dense layer with its rotation kept in factors)
     had_block: int        # block size of the block-diagonal Hadamard (0 for dense)
     nu: float = 4.0
     w_std: float = 0.02
@@ -114,6 +152,15 @@ class LayerSpec:
         if self.rot != "dense":
             return None
         return f32_to_bf16_bits(make_orthogonal(self.seed, self.K).astype(np.float32))
+
+
+    def dual_factors(self, Bd: int = 128):
+        """(Bd, R1 bf16 bits [K/Bd,Bd,Bd], perm int32 [K], R2 bf16 bits [K/Bd,Bd,Bd]) of a seeded dual transformation
+        y = x . blockdiag(R1) . P . blockdiag(R2); the permutation leads with this layer's salient channels."""
+        R1 = f32_to_bf16_bits(make_block_rotations(self.seed, self.K, Bd).astype(np.float32))
+        R2 = f32_to_bf16_bits(make_block_rotations(self.seed + 7, self.K, Bd).astype(np.float32))
+        perm = make_staggered_permutation(self.seed, self.K, Bd, salient_channels(self.seed, self.K, self.n_salient))
+        return Bd, R1, perm, R2
 
 
 def _largest_pow2_divisor(k: int) -> int:

@@ -120,6 +120,58 @@ int orc_rotate_dense(const double *X, int M, int K, const double *R, double *Y) 
     return 0;
 }
 
+/* Sec. 4.2, the dual transformation behind the second case of Eq. 12, kept in its factors:
+ *   y = x . R1hat . P . R2hat
+ * R1hat, R2hat block-diagonal with K/Bd orthogonal blocks of Bd x Bd (block j row-major at R[j*Bd*Bd],
+ * acting on channels j*Bd .. j*Bd+Bd-1: u_{jBd+i} = sum_l x_{jBd+l} R[j][l][i]); P the channel
+ * reordering, given as an index map: (u . P)_i = u_{perm[i]}, i.e. P[l][i] = 1 exactly when l = perm[i].
+ * The three maps are applied one after the other, each sum over l in increasing order.
+ * Returns -1 when Bd does not divide K or perm is not a permutation of 0..K-1. */
+int orc_rotate_dual(const double *X, int M, int K, int Bd, const double *R1, const int32_t *perm,
+                    const double *R2, double *Y) {
+    if (Bd < 1 || K % Bd) return -1;
+    {
+        char *seen = (char *)calloc((size_t)K, 1);
+        int bad = 0;
+        for (int i = 0; i < K; ++i) {
+            if (perm[i] < 0 || perm[i] >= K || seen[perm[i]]) { bad = 1; break; }
+            seen[perm[i]] = 1;
+        }
+        free(seen);
+        if (bad) return -1;
+    }
+#pragma omp parallel
+    {
+        double *u = (double *)malloc((size_t)K * sizeof(double));
+        double *v = (double *)malloc((size_t)K * sizeof(double));
+#pragma omp for schedule(static)
+        for (int m = 0; m < M; ++m) {
+            const double *x = X + (size_t)m * K;
+            double *y = Y + (size_t)m * K;
+            for (int j = 0; j < K / Bd; ++j) {             /* u = x . R1hat */
+                const double *Rj = R1 + (size_t)j * Bd * Bd;
+                for (int i = 0; i < Bd; ++i) {
+                    double acc = 0.0;
+                    for (int l = 0; l < Bd; ++l) acc += x[j * Bd + l] * Rj[(size_t)l * Bd + i];
+                    u[j * Bd + i] = acc;
+                }
+            }
+            for (int i = 0; i < K; ++i) v[i] = u[perm[i]]; /* v = u . P */
+            for (int j = 0; j < K / Bd; ++j) {             /* y = v . R2hat */
+                const double *Rj = R2 + (size_t)j * Bd * Bd;
+                for (int i = 0; i < Bd; ++i) {
+                    double acc = 0.0;
+                    for (int l = 0; l < Bd; ++l) acc += v[j * Bd + l] * Rj[(size_t)l * Bd + i];
+                    y[j * Bd + i] = acc;
+                }
+            }
+        }
+        free(u);
+        free(v);
+    }
+    return 0;
+}
+
 static double clampd(double v, double lo, double hi) { return v < lo ? lo : (v > hi ? hi : v); }
 
 /* ------------------------------------------------------------------------------------------

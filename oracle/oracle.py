@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "liblrq_oracle.so")
 
 __all__ = [
     "build", "num_threads", "hadamard_matrix", "rotate_hadamard_explicit", "rotate_hadamard_fwht",
-    "rotate_dense", "quantize_act", "dequantize_act", "level_value", "tlq_quantize", "qmatmul",
+    "rotate_dense", "rotate_dual", "quantize_act", "dequantize_act", "level_value", "tlq_quantize", "qmatmul",
     "TLQResult", "qlinear", "smooth", "fluctuation_metric", "rotate_weights",
 ]
 
@@ -99,6 +99,23 @@ def rotate_dense(X, R):
     return Y
 
 
+def rotate_dual(X, Bd: int, R1, perm, R2):
+    """y = x . R1hat . P . R2hat, the dual transformation of Sec. 4.2 in its factors: R1hat and R2hat
+    block-diagonal with blocks R1[j], R2[j] of Bd x Bd (arrays [K/Bd, Bd, Bd]); P as the index map
+    (u P)_i = u[perm[i]]."""
+    X, xp = _d(X)
+    R1, r1p = _d(R1)
+    R2, r2p = _d(R2)
+    M, K = X.shape
+    perm = np.ascontiguousarray(perm, dtype=np.int32)
+    assert K % Bd == 0 and R1.shape == (K // Bd, Bd, Bd) and R2.shape == R1.shape and perm.shape == (K,)
+    Y = np.empty_like(X)
+    rc = _L().orc_rotate_dual(xp, M, K, int(Bd), r1p, perm.ctypes.data_as(_ip), r2p, Y.ctypes.data_as(_dp))
+    if rc:
+        raise ValueError("Bd must divide K and perm must be a permutation of range(K)")
+    return Y
+
+
 def smooth(X, p):
     """X diag(p): the channel-wise smoothing multipliers applied to the activations (Sec. 5.1)."""
     X, xp = _d(X)
@@ -110,7 +127,7 @@ def smooth(X, p):
     return Y
 
 
-def rotate_weights(W, colmul=None, rot: str = "hadamard", had_block: int = 0, R=None):
+def rotate_weights(W, colmul=None, rot: str = "hadamard", had_block: int = 0, R=None, dual=None):
     """The weight side of Eq. 2, (X R)(W R)^T = X W^T: the rows of W diag(colmul) mapped by the layer's rotation
     (Sec. 3.2; colmul is the reciprocal of the activations' smoothing multipliers, Sec. 5.1).  The same maps the
     activations take, applied to weight rows."""
@@ -121,6 +138,8 @@ def rotate_weights(W, colmul=None, rot: str = "hadamard", had_block: int = 0, R=
         return rotate_hadamard_fwht(W, had_block)
     if rot == "dense":
         return rotate_dense(W, R)
+    if rot == "dual":
+        return rotate_dual(W, *dual)
     if rot == "none":
         return W.copy()
     raise ValueError(rot)
@@ -224,7 +243,7 @@ def qmatmul(Q, S, Z, tlq: TLQResult, wscale=None, bias=None):
 
 
 def qlinear(X, tlq: TLQResult, a_bits: int, rot: str, had_block: int = 0, R=None, mode: int = 0,
-            wscale=None, bias=None, prescale=None, return_rotated: bool = False):
+            wscale=None, bias=None, prescale=None, return_rotated: bool = False, dual=None):
     """The whole layer on already-widened inputs: [smooth (Sec. 5.1) ->] rotate (Eq. 12) -> per-token
     quantize (Eq. 1) -> contraction with the TLQ table and epilogue (Eq. 10).  Returns (Y, codes, s, z), and with
     return_rotated also the rotated activations that Eq. 1 quantized."""
@@ -234,6 +253,8 @@ def qlinear(X, tlq: TLQResult, a_bits: int, rot: str, had_block: int = 0, R=None
         Yr = rotate_hadamard_fwht(X, had_block)
     elif rot == "dense":
         Yr = rotate_dense(X, R)
+    elif rot == "dual":
+        Yr = rotate_dual(X, *dual)                     # dual = (Bd, R1, perm, R2)
     elif rot == "none":
         Yr = np.ascontiguousarray(X, dtype=np.float64)
     else:

@@ -22,9 +22,8 @@ EXPORTS = [
     "lrq_tlq_quantize_weights", "lrq_act_workspace_bytes", "lrq_rotate_quantize_act", "lrq_layer_create",
     "lrq_layer_destroy", "lrq_workspace_bytes", "lrq_qlinear", "lrq_qlinear_stack", "lrq_qgemm_codes",
     "lrq_device_status", "lrq_status_string", "lrq_version", "lrq_rotate_quantize_act_static", "lrq_ars_select",
-    "lrq_rotate_weights", "lrq_selftest_wait_timeout",
+    "lrq_rotate_weights", "lrq_selftest_wait_timeout", "lrq_static_scratch_bytes",
 ]
-STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class LrqError(RuntimeError):
@@ -79,6 +78,8 @@ def load_library() -> C.CDLL:
     lib.lrq_selftest_wait_timeout.argtypes = [C.c_longlong, vp]
     lib.lrq_status_string.argtypes = [ci]
     lib.lrq_status_string.restype = C.c_char_p
+    lib.lrq_static_scratch_bytes.argtypes = []
+    lib.lrq_static_scratch_bytes.restype = sz
     for name in EXPORTS:
         getattr(lib, name)
     _lib = lib
@@ -120,6 +121,11 @@ def lrq_selftest_wait_timeout(limit_cycles: int = 100000, stream=None) -> None:
 
 
 SELFTEST_WAIT_CODE = 99
+
+
+def lrq_static_scratch_bytes() -> int:
+    """Size of the fixed scratch array behind lrq_rotate_quantize_act_static, as built into the library."""
+    return int(load_library().lrq_static_scratch_bytes())
 
 
 # ------------------------------------------------------------------------------------------------
@@ -231,7 +237,7 @@ def lrq_rotate_quantize_act_static(X: torch.Tensor, kind: int, a_bits: int, had_
                                    R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM, stream=None, out=None):
     """lrq_rotate_quantize_act for callers that cannot provide device scratch (a host that may not call
     cudaMalloc once it is running, or whose memory is planned by another runtime): the dense rotation's
-    scratch is a fixed STATIC_SCRATCH_BYTES array inside the library.  ``out`` (codes, scale, zero_point)
+    scratch is a fixed array of lrq_static_scratch_bytes() bytes inside the library.  ``out`` (codes, scale, zero_point)
     lets such a caller pass its own pre-planned result buffers; without it this wrapper allocates them with
     torch, the C entry point itself never allocates.  Raises LrqError (workspace) when M*K*4 exceeds the array."""
     _need_cuda(X, R)

@@ -94,28 +94,21 @@ extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long 
 // ---------------------------------------------------------------------------------------------------
 // Variant for callers that cannot allocate: the dense rotation's fp32 scratch is this fixed array.
 // In host code `g_static_scratch` is only a handle to the symbol; its address on the current device
-// comes from cudaGetSymbolAddress, queried once per device and cached.
+// comes from cudaGetSymbolAddress.  The address is asked for on every call (a host-side table lookup once
+// the module is loaded) rather than cached, so that it stays right after the application resets a device.
 // ---------------------------------------------------------------------------------------------------
 static __device__ __align__(256) unsigned char g_static_scratch[LRQ_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
-std::mutex g_scratch_mutex;
-void* g_scratch_addr[kMaxDevices] = {};
-
 // Device address of the static scratch on the current device (nullptr on failure).
 void* static_scratch_address() {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return nullptr; }
-    std::lock_guard<std::mutex> lock(g_scratch_mutex);
-    if (!g_scratch_addr[dev]) {
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
-        g_scratch_addr[dev] = ptr;
-    }
-    return g_scratch_addr[dev];
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return ptr;
 }
 }  // namespace
+
+extern "C" size_t lrq_static_scratch_bytes(void) { return (size_t)LRQ_STATIC_SCRATCH_BYTES; }
 
 extern "C" lrq_status lrq_rotate_quantize_act_static(const void* X, int M, int K, long ldx, const lrq_act_params* p,
                                                      uint8_t* a_codes, float* a_scale, int32_t* a_zp,

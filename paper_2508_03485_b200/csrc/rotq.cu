@@ -1,10 +1,15 @@
 // Rotation + per-token activation quantization (Sec. 4.2 Eq. 12, first case; Sec. 3.1 Eq. 1).
 //
 // HBM-bound step: each activation is read once (bf16) and written once as a 4- or 8-bit code.
-// The block-diagonal Walsh-Hadamard transform runs in fp32: three butterfly stages in registers
-// on the 8 elements of one 128-bit load, the remaining stages three at a time through shared
-// memory.  The 1/sqrt(B) normalisation is never applied to the elements: it is folded into the
-// per-token scale, since rint(y/s) is invariant under a common factor of y and s.
+// This file holds the register-resident kernels: a thread keeps 8 consecutive channels of a token (16 with
+// 256-bit loads), runs the first butterfly stages of the block-diagonal Walsh-Hadamard transform on them in
+// fp32, the next stages by warp shuffles, and for blocks above 256 the rest through one shared-memory
+// transpose; the per-token range is reduced with redux.sync and one named barrier, and the kernel is
+// persistent with the next token group's loads in flight.  Blocks of 8..128 with K a multiple of 128 go to the
+// TMA-fed kernel of rotq_blk.cu first; a generic shared-memory kernel covers whatever neither takes.
+// The 1/sqrt(B) normalisation is never applied to the elements: it is folded into the per-token scale, since
+// rint(y/s) is invariant under a common factor of y and s.  The fp32 quantizer after a dense rotation and the
+// fluctuation metric of Eq. 11 live here as well.
 #include "lrq_internal.cuh"
 #include "f32x2.cuh"
 #include "rotq_common.cuh"

@@ -118,3 +118,74 @@ def test_rotation_invariance_of_the_product(orc):
     ref = X @ W.T
     for rot in (lambda A: orc.rotate_hadamard_fwht(A, 64), lambda A: orc.rotate_dense(A, make_orthogonal(1, K))):
         assert np.abs(rot(X) @ rot(W).T - ref).max() < 1e-12
+
+
+# ------------------------------------------------------------------ the dual transformation in its factors (Sec. 4.2)
+def _dual_inputs(K=256, Bd=64, seed=3):
+    from lrq_workloads import make_block_rotations, make_staggered_permutation
+    R1 = make_block_rotations(seed, K, Bd)
+    R2 = make_block_rotations(seed + 1, K, Bd)
+    perm = make_staggered_permutation(seed, K, Bd, np.array([5, 70, 7, 200]))
+    return R1, perm, R2
+
+
+def test_dual_rotation_worked_example(orc):
+    # K = 4, blocks of 2, worked by hand: u = x R1 = [-2, 1, 3, 4]; v_i = u[perm[i]] = [3, -2, 4, 1];
+    # y = v R2 = [2, 3, 1, -4].  A transposed block or a scatter instead of a gather gives other numbers.
+    q = np.array([[0.0, 1.0], [-1.0, 0.0]])                       # x q = [-x1, x0]
+    R1 = np.stack([q, np.eye(2)])
+    R2 = np.stack([q, q.T])
+    y = orc.rotate_dual(np.array([[1.0, 2.0, 3.0, 4.0]]), 2, R1, [2, 0, 3, 1], R2)
+    assert np.array_equal(y, [[2.0, 3.0, 1.0, -4.0]])
+
+
+def test_dual_rotation_equals_dense_rotation_by_the_composed_matrix(orc):
+    K, Bd = 256, 64
+    R1, perm, R2 = _dual_inputs(K, Bd)
+    Pm = np.zeros((K, K))
+    Pm[perm, np.arange(K)] = 1.0                                  # (u P)_i = u[perm[i]]
+    R = scipy.linalg.block_diag(*R1) @ Pm @ scipy.linalg.block_diag(*R2)
+    assert np.abs(R @ R.T - np.eye(K)).max() < 1e-12              # the composition is a rotation
+    X = np.random.default_rng(0).standard_normal((9, K)) * 4.0
+    Yd = orc.rotate_dual(X, Bd, R1, perm, R2)
+    assert np.abs(Yd - orc.rotate_dense(X, R)).max() < 1e-12
+    assert np.abs(Yd - X @ R).max() < 1e-12
+    assert np.allclose(np.linalg.norm(Yd, axis=1), np.linalg.norm(X, axis=1), rtol=1e-13)   # Lemma 1: norms kept
+
+
+def test_dual_rotation_special_cases(orc):
+    K, Bd = 256, 64
+    R1, perm, R2 = _dual_inputs(K, Bd)
+    X = np.random.default_rng(1).standard_normal((5, K))
+    eye = np.broadcast_to(np.eye(Bd), R1.shape)
+    ident = np.arange(K)
+    # R2 = I, P = I: the blocks of R1 act on their own channels only
+    Y = orc.rotate_dual(X, Bd, R1, ident, eye)
+    assert np.abs(Y - np.einsum("mjl,jli->mji", X.reshape(5, K // Bd, Bd), R1).reshape(5, K)).max() < 1e-13
+    # R1 = R2 = I: a pure reordering, exactly
+    assert np.array_equal(orc.rotate_dual(X, Bd, eye, perm, eye), X[:, perm])
+    # one block of K channels and no reordering: two dense rotations in a row
+    Q1 = _dual_inputs(K, K, 8)[0]
+    Q2 = _dual_inputs(K, K, 9)[0]
+    assert np.abs(orc.rotate_dual(X, K, Q1, ident, Q2) - X @ Q1[0] @ Q2[0]).max() < 1e-12
+
+
+def test_dual_rotation_spreads_leading_channels_over_blocks():
+    from lrq_workloads import make_staggered_permutation
+    K, Bd = 1152, 128
+    first = np.array([3, 4, 5, 6, 7, 8, 9, 10, 11, 600])          # nine neighbours of one block, and one more
+    perm = make_staggered_permutation(0, K, Bd, first)
+    assert np.array_equal(np.sort(perm), np.arange(K))
+    where = {int(c): i // Bd for i, c in enumerate(perm)}
+    assert sorted(where[int(c)] for c in first[:9]) == list(range(9))   # one per block
+    assert where[600] == 8                                        # the second pass runs backwards
+
+
+def test_dual_rotation_rejects_a_non_permutation(orc):
+    R1, perm, R2 = _dual_inputs()
+    bad = perm.copy()
+    bad[0] = bad[1]
+    with pytest.raises(ValueError):
+        orc.rotate_dual(np.zeros((1, 256)), 64, R1, bad, R2)
+    with pytest.raises(ValueError):
+        orc.rotate_dual(np.zeros((1, 256)), 64, R1, np.arange(256) + 1, R2)

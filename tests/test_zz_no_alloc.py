@@ -23,15 +23,32 @@ def P():
     return P
 
 
+def _free_bytes():
+    return torch.cuda.mem_get_info()[0]
+
+
 def test_static_scratch_matches_workspace_path_twice(P):
     K = 384
     R = PU.bf16_to_device(f32_to_bf16_bits(make_orthogonal(11, K).astype(np.float32)))
+    warm = PU.bf16_to_device(make_activations(9, 1, K))
+    P.lrq_rotate_quantize_act_static(warm, P.ROT_DENSE, 8, R=R)                # start-up call: loads the module
+    torch.cuda.synchronize()
     # second call: fewer tokens and other data, so stale scratch rows from the first call lie beyond it
     for M, seed, a_bits in [(300, 1, 8), (77, 2, 4)]:
         X = PU.bf16_to_device(make_activations(seed, M, K, n_salient=16, salient_x=100.0))
         ref = P.lrq_rotate_quantize_act(X, P.ROT_DENSE, a_bits, R=R)
-        got = P.lrq_rotate_quantize_act_static(X, P.ROT_DENSE, a_bits, R=R)
+        # the caller's own result buffers, as a host that may not allocate would pass them
+        out = (torch.empty((M, K * a_bits // 8), dtype=torch.uint8, device="cuda"),
+               torch.empty((M,), dtype=torch.float32, device="cuda"),
+               torch.empty((M,), dtype=torch.int32, device="cuda"))
         torch.cuda.synchronize()
+        held, reserved, free = torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), _free_bytes()
+        got = P.lrq_rotate_quantize_act_static(X, P.ROT_DENSE, a_bits, R=R, out=out)
+        torch.cuda.synchronize()
+        # nothing was allocated: neither through torch's allocator nor behind its back on the device
+        assert torch.cuda.memory_allocated() == held and torch.cuda.memory_reserved() == reserved
+        assert _free_bytes() == free
+        assert all(g is o for g, o in zip(got, out))
         for g, r in zip(got, ref):
             assert torch.equal(g, r)
     assert P.lrq_device_status() == 0
@@ -46,7 +63,7 @@ def test_static_scratch_other_kinds_and_limit(P):
         assert torch.equal(g, r)
     # one token too many for the fixed array: refused with the workspace status, nothing launched
     K = 1024
-    M = P.STATIC_SCRATCH_BYTES // (4 * K) + 1
+    M = P.lrq_static_scratch_bytes() // (4 * K) + 1
     Xb = torch.zeros((M, K), dtype=torch.bfloat16, device="cuda")
     Rb = torch.zeros((K, K), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(P.LrqError) as e:
