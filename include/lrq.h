@@ -43,7 +43,7 @@ typedef enum {
     LRQ_ERR_TIMEOUT = 5        /* a bounded device-side wait expired                               */
 } lrq_status;
 
-typedef enum { LRQ_ROT_NONE = 0, LRQ_ROT_HADAMARD = 1, LRQ_ROT_DENSE = 2 } lrq_rot_kind;
+typedef enum { LRQ_ROT_NONE = 0, LRQ_ROT_HADAMARD = 1, LRQ_ROT_DENSE = 2, LRQ_ROT_DUAL = 3 } lrq_rot_kind;
 typedef enum { LRQ_ACT_ASYM = 0, LRQ_ACT_SYM = 1 } lrq_act_mode;
 typedef enum { LRQ_F32 = 0, LRQ_F16 = 1, LRQ_BF16 = 2 } lrq_dtype;
 /* Storage of the weight codes (Sec. 4.1, Eq. 5: a b-bit code per weight).
@@ -95,6 +95,12 @@ lrq_status lrq_tlq_quantize_weights(const float* W_rot, int N, int K, const lrq_
  *             a power of two (8..4096) dividing K: one fused kernel, fp32 butterflies.
  *   DENSE     y = x . R with the composed outlier-aware rotation given as one bf16 K x K matrix
  *             (second case of Eq. 12): a tcgen05 GEMM into an fp32 scratch, then the quantizer.
+ *   DUAL      the same outlier-aware transformation kept in the factors Sec. 4.2 builds it from,
+ *             y = x . R1hat . P . R2hat: R1hat, R2hat block-diagonal with K/Bd orthogonal bf16 blocks of
+ *             Bd x Bd, P the staggered channel reordering as an index map, (u P)_i = u[perm[i]].  Two
+ *             block-diagonal tcgen05 products (2.M.K.Bd flop each instead of 2.M.K.K, and no K x K matrix to
+ *             read) with a gather between them; the gathered fp32 intermediate is split into three bf16 terms
+ *             so that the second product keeps fp32 accuracy.  Bd = 128, K a multiple of 128.
  *   NONE      y = x.
  * then, per token, ASYM: s = (max-min)/(2^b-1), z = rint(min/s), q = clamp(rint(y/s)-z, 0, 2^b-1);
  *                  SYM : s = max|y|/(2^(b-1)-1), z = -2^(b-1), same q.   Rounding is to nearest even.
@@ -108,10 +114,18 @@ typedef struct {
     const float* prescale;   /* nullable dev float [K], 16-byte aligned: smoothing multipliers applied
                                 channel-wise before the rotation (Sec. 5.1: X' = X diag(prescale), the
                                 weights having absorbed diag(1/prescale)).  HADAMARD / NONE only; for a
-                                DENSE rotation fold diag(prescale) into R.                            */
+                                DENSE or DUAL rotation fold diag(prescale) into R / R1.               */
+    /* DUAL only (ignored otherwise): */
+    int dual_block;          /* Bd: 128                                                            */
+    const void* R1_bf16;     /* dev bf16 [K/Bd,Bd,Bd]: u_{jBd+i} = sum_l x_{jBd+l} R1[j][l][i]; 16-byte aligned */
+    const int32_t* perm;     /* dev int32 [K]: a permutation of 0..K-1; position i takes channel perm[i].  An entry
+                                outside 0..K-1 is read as channel 0 and recorded (lrq_device_status code 31).  */
+    const void* R2_bf16;     /* dev bf16 [K/Bd,Bd,Bd], applied after the reordering                */
 } lrq_act_params;
 
-/* Bytes of workspace lrq_rotate_quantize_act needs for M tokens (0 unless kind == DENSE). */
+/* Bytes of workspace lrq_rotate_quantize_act needs for M tokens: 0 for HADAMARD / NONE, 4.M.K for DENSE (the fp32
+ * rotated activations), 10.M.K for DUAL (an fp32 array that holds first u, later y, and the three bf16 terms of
+ * the reordered u). */
 size_t lrq_act_workspace_bytes(int M, int K, const lrq_act_params* p);
 
 /*
@@ -153,6 +167,12 @@ lrq_status lrq_ars_select(const void* X_bf16, int M, int K, long ldx, double thr
 lrq_status lrq_rotate_weights(const float* W, int N, int K, long ldw, const float* colmul, lrq_rot_kind kind,
                               int had_block, const void* R_bf16, float* W_rot, long ldo, void* cuda_stream);
 
+/* The same for the dual transformation in its factors (LRQ_ROT_DUAL): W_rot = W diag(colmul) R1hat P R2hat,
+ * arguments as in lrq_act_params.  Each row is held in shared memory as fp64: K <= 12288. */
+lrq_status lrq_rotate_weights_dual(const float* W, int N, int K, long ldw, const float* colmul, int dual_block,
+                                   const void* R1_bf16, const int32_t* perm, const void* R2_bf16,
+                                   float* W_rot, long ldo, void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------------------
  * lrq_rotate_quantize_act for callers that cannot hand over device scratch.
  *
@@ -167,9 +187,9 @@ lrq_status lrq_rotate_weights(const float* W, int N, int K, long ldw, const floa
  * (LRQ_STATIC_SCRATCH_BYTES, held by every GPU that loads the library until the process exits).
  *
  *   - Arguments and results are those of lrq_rotate_quantize_act without the workspace pair.
- *   - kind == LRQ_ROT_DENSE needs M*K*4 <= LRQ_STATIC_SCRATCH_BYTES, otherwise the call returns
- *     LRQ_ERR_WORKSPACE and launches nothing (split the tokens into several calls).  The other
- *     kinds use no scratch and have no size limit.
+ *   - kind == LRQ_ROT_DENSE needs M*K*4 <= LRQ_STATIC_SCRATCH_BYTES (LRQ_ROT_DUAL: M*K*10), otherwise the
+ *     call returns LRQ_ERR_WORKSPACE and launches nothing (split the tokens into several calls).  The
+ *     other kinds use no scratch and have no size limit.
  *   - The call allocates nothing (no cudaMalloc/cudaFree, no allocating library routine).  Every call
  *     asks the runtime for the device address of the array (a host-side query, no launch, nothing cached
  *     here, so a device reset between calls is harmless).  The FIRST call of the process on each device

@@ -8,5 +8,6 @@ from .binding import (  # noqa: F401
     StackPlan, lrq_rotate_quantize_act_static, lrq_static_scratch_bytes,
     load_library, LrqError, TLQWeights, QLayer,
     lrq_tlq_quantize_weights, lrq_rotate_quantize_act, lrq_qlinear, lrq_qlinear_stack, lrq_qgemm_codes,
-    lrq_ars_select, lrq_rotate_weights, lrq_device_status, lrq_version, ROT_NONE, ROT_HADAMARD, ROT_DENSE, ACT_ASYM, ACT_SYM, F32, F16, BF16, CODES_NIBBLE, CODES_PACKED3, lrq_selftest_wait_timeout, SELFTEST_WAIT_CODE,
+    lrq_ars_select, lrq_rotate_weights, lrq_device_status, lrq_version, ROT_NONE, ROT_HADAMARD, ROT_DENSE, ROT_DUAL,
+    DualRotation, lrq_rotate_weights_dual, ACT_ASYM, ACT_SYM, F32, F16, BF16, CODES_NIBBLE, CODES_PACKED3, lrq_selftest_wait_timeout, SELFTEST_WAIT_CODE,
 )

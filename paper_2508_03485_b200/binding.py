@@ -12,7 +12,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIBPATH = os.path.join(_HERE, "liblrq_b200.so")
 
-ROT_NONE, ROT_HADAMARD, ROT_DENSE = 0, 1, 2
+ROT_NONE, ROT_HADAMARD, ROT_DENSE, ROT_DUAL = 0, 1, 2, 3
 ACT_ASYM, ACT_SYM = 0, 1
 F32, F16, BF16 = 0, 1, 2
 CODES_NIBBLE, CODES_PACKED3 = 0, 1
@@ -22,7 +22,7 @@ EXPORTS = [
     "lrq_tlq_quantize_weights", "lrq_act_workspace_bytes", "lrq_rotate_quantize_act", "lrq_layer_create",
     "lrq_layer_destroy", "lrq_workspace_bytes", "lrq_qlinear", "lrq_qlinear_stack", "lrq_qgemm_codes",
     "lrq_device_status", "lrq_status_string", "lrq_version", "lrq_rotate_quantize_act_static", "lrq_ars_select",
-    "lrq_rotate_weights", "lrq_selftest_wait_timeout", "lrq_static_scratch_bytes",
+    "lrq_rotate_weights", "lrq_selftest_wait_timeout", "lrq_static_scratch_bytes", "lrq_rotate_weights_dual",
 ]
 
 
@@ -41,7 +41,8 @@ class _TlqParams(C.Structure):
 
 class _ActParams(C.Structure):
     _fields_ = [("kind", C.c_int), ("had_block", C.c_int), ("R_bf16", C.c_void_p),
-                ("a_bits", C.c_int), ("mode", C.c_int), ("prescale", C.c_void_p)]
+                ("a_bits", C.c_int), ("mode", C.c_int), ("prescale", C.c_void_p),
+                ("dual_block", C.c_int), ("R1_bf16", C.c_void_p), ("perm", C.c_void_p), ("R2_bf16", C.c_void_p)]
 
 
 _lib = None
@@ -74,6 +75,7 @@ def load_library() -> C.CDLL:
     lib.lrq_qgemm_codes.argtypes = [vp, vp, vp, vp, ci, vp, ci, cl, ci, vp]
     lib.lrq_ars_select.argtypes = [vp, ci, ci, cl, C.c_double, vp, vp, vp, sz, vp]
     lib.lrq_rotate_weights.argtypes = [vp, ci, ci, cl, vp, ci, ci, vp, vp, cl, vp]
+    lib.lrq_rotate_weights_dual.argtypes = [vp, ci, ci, cl, vp, ci, vp, vp, vp, vp, cl, vp]
     lib.lrq_device_status.argtypes = [vp]
     lib.lrq_selftest_wait_timeout.argtypes = [C.c_longlong, vp]
     lib.lrq_status_string.argtypes = [ci]
@@ -163,12 +165,49 @@ def lrq_tlq_quantize_weights(W_rot: torch.Tensor, w_bits: int, group_size: int =
     return TLQWeights(codes, levels, meta, wsum, int(w_bits), int(group_size), int(code_layout))
 
 
+@dataclass
+class DualRotation:
+    """The dual transformation of Sec. 4.2 in its factors, y = x . blockdiag(R1) . P . blockdiag(R2)."""
+    block: int             # Bd
+    R1: torch.Tensor       # bfloat16 [K/Bd, Bd, Bd]
+    perm: torch.Tensor     # int32 [K]: position i takes channel perm[i]
+    R2: torch.Tensor       # bfloat16 [K/Bd, Bd, Bd]
+
+    def check(self, K: int):
+        nb = K // self.block
+        for R in (self.R1, self.R2):
+            assert R.is_cuda and R.dtype == torch.bfloat16 and R.shape == (nb, self.block, self.block) and R.is_contiguous()
+        assert self.perm.is_cuda and self.perm.dtype == torch.int32 and self.perm.shape == (K,) and self.perm.is_contiguous()
+
+
 def _act_params(kind: int, had_block: int, R: Optional[torch.Tensor], a_bits: int, mode: int,
-                prescale: Optional[torch.Tensor] = None) -> _ActParams:
+                prescale: Optional[torch.Tensor] = None, dual: Optional[DualRotation] = None) -> _ActParams:
     if prescale is not None:
         assert prescale.dtype == torch.float32 and prescale.is_contiguous()
-    return _ActParams(int(kind), int(had_block), 0 if R is None else R.data_ptr(), int(a_bits), int(mode),
-                      0 if prescale is None else prescale.data_ptr())
+    p = _ActParams(int(kind), int(had_block), 0 if R is None else R.data_ptr(), int(a_bits), int(mode),
+                   0 if prescale is None else prescale.data_ptr(), 0, 0, 0, 0)
+    if dual is not None:
+        p.dual_block, p.R1_bf16, p.perm, p.R2_bf16 = int(dual.block), dual.R1.data_ptr(), dual.perm.data_ptr(), dual.R2.data_ptr()
+    return p
+
+
+def lrq_rotate_weights_dual(W: torch.Tensor, dual: DualRotation, colmul: Optional[torch.Tensor] = None, stream=None,
+                            out: Optional[torch.Tensor] = None):
+    """W diag(colmul) R1hat P R2hat in fp64, rounded to fp32: the weight side of Eq. 2 for a layer whose rotation is kept
+    in the factors of the dual transformation.  Returns W_rot float32 [N,K]."""
+    _need_cuda(W)
+    assert W.dtype == torch.float32 and W.dim() == 2 and W.stride(1) == 1
+    N, K = W.shape
+    dual.check(K)
+    if colmul is not None:
+        assert colmul.dtype == torch.float32 and colmul.shape == (K,) and colmul.is_contiguous()
+    if out is None:
+        out = torch.empty((N, K), dtype=torch.float32, device=W.device)
+    assert out.dtype == torch.float32 and out.shape == (N, K) and out.stride(1) == 1
+    _check(load_library().lrq_rotate_weights_dual(_ptr(W), N, K, W.stride(0), _ptr(colmul), dual.block, _ptr(dual.R1),
+                                                  _ptr(dual.perm), _ptr(dual.R2), _ptr(out), out.stride(0),
+                                                  _stream(stream)), "lrq_rotate_weights_dual")
+    return out
 
 
 def lrq_rotate_weights(W: torch.Tensor, kind: int, had_block: int = 0, R: Optional[torch.Tensor] = None,
@@ -207,14 +246,16 @@ def lrq_ars_select(X: torch.Tensor, threshold: float = 1.0, stream=None):
 def lrq_rotate_quantize_act(X: torch.Tensor, kind: int, a_bits: int, had_block: int = 0,
                             R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM,
                             workspace: Optional[torch.Tensor] = None, stream=None, out=None,
-                            prescale: Optional[torch.Tensor] = None):
+                            prescale: Optional[torch.Tensor] = None, dual: Optional[DualRotation] = None):
     """Rotation + per-token quantization (Eq. 12, Eq. 1) of device bf16 [M,K] activations.
     Returns (codes uint8, scale float32 [M], zero_point int32 [M])."""
     _need_cuda(X, R, workspace, prescale)
     assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
     M, K = X.shape
     lib = load_library()
-    p = _act_params(kind, had_block, R, a_bits, mode, prescale)
+    if dual is not None:
+        dual.check(K)
+    p = _act_params(kind, had_block, R, a_bits, mode, prescale, dual)
     need = int(lib.lrq_act_workspace_bytes(M, K, C.byref(p)))
     if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
         workspace = torch.empty(need, dtype=torch.uint8, device=X.device)
@@ -234,7 +275,8 @@ def lrq_rotate_quantize_act(X: torch.Tensor, kind: int, a_bits: int, had_block: 
 
 
 def lrq_rotate_quantize_act_static(X: torch.Tensor, kind: int, a_bits: int, had_block: int = 0,
-                                   R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM, stream=None, out=None):
+                                   R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM, stream=None, out=None,
+                                   dual: Optional[DualRotation] = None):
     """lrq_rotate_quantize_act for callers that cannot provide device scratch (a host that may not call
     cudaMalloc once it is running, or whose memory is planned by another runtime): the dense rotation's
     scratch is a fixed array of lrq_static_scratch_bytes() bytes inside the library.  ``out`` (codes, scale, zero_point)
@@ -249,7 +291,9 @@ def lrq_rotate_quantize_act_static(X: torch.Tensor, kind: int, a_bits: int, had_
         codes = torch.empty((M, K * a_bits // 8), dtype=torch.uint8, device=X.device)
         scale = torch.empty((M,), dtype=torch.float32, device=X.device)
         zp = torch.empty((M,), dtype=torch.int32, device=X.device)
-    p = _act_params(kind, had_block, R, a_bits, mode)
+    if dual is not None:
+        dual.check(K)
+    p = _act_params(kind, had_block, R, a_bits, mode, None, dual)
     rc = load_library().lrq_rotate_quantize_act_static(_ptr(X), M, K, X.stride(0), C.byref(p), _ptr(codes),
                                                        _ptr(scale), _ptr(zp), _stream(stream))
     _check(rc, "lrq_rotate_quantize_act_static")
@@ -262,12 +306,14 @@ class QLayer:
     def __init__(self, tlq: TLQWeights, N: int, K: int, kind: int, a_bits: int, had_block: int = 0,
                  R: Optional[torch.Tensor] = None, mode: int = ACT_ASYM,
                  wscale: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
-                 prescale: Optional[torch.Tensor] = None):
+                 prescale: Optional[torch.Tensor] = None, dual: Optional[DualRotation] = None):
         _need_cuda(tlq.codes, tlq.levels, tlq.wsum, R, wscale, bias, prescale)
-        self.prescale = prescale
+        if dual is not None:
+            dual.check(K)
+        self.prescale, self.dual = prescale, dual
         self.tlq, self.N, self.K, self.R, self.wscale, self.bias = tlq, N, K, R, wscale, bias
         self.kind, self.a_bits, self.had_block, self.mode = kind, a_bits, had_block, mode
-        self._p = _act_params(kind, had_block, R, a_bits, mode, prescale)
+        self._p = _act_params(kind, had_block, R, a_bits, mode, prescale, dual)
         h = C.c_void_p()
         rc = load_library().lrq_layer_create(C.byref(h), N, K, tlq.w_bits, tlq.group, tlq.code_layout, _ptr(tlq.codes),
                                              _ptr(tlq.levels), _ptr(tlq.wsum), _ptr(wscale), _ptr(bias),

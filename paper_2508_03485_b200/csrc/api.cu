@@ -58,6 +58,12 @@ static lrq_status check_act(const lrq_act_params* p, int K) {
             if (!lrq_aligned(p->R_bf16, 16)) return LRQ_ERR_INVALID_ARG;
             if (p->prescale) return LRQ_ERR_UNSUPPORTED;      // fold diag(prescale) into R instead
             break;
+        case LRQ_ROT_DUAL:
+            if (!p->R1_bf16 || !p->R2_bf16 || !p->perm) return LRQ_ERR_INVALID_ARG;
+            if (!lrq_aligned(p->R1_bf16, 16) || !lrq_aligned(p->R2_bf16, 16) || !lrq_aligned(p->perm, 4)) return LRQ_ERR_INVALID_ARG;
+            if (p->dual_block != 128 || K % 128 || K > 12288) return LRQ_ERR_UNSUPPORTED;
+            if (p->prescale) return LRQ_ERR_UNSUPPORTED;      // fold diag(prescale) into R1 instead
+            break;
         default: return LRQ_ERR_INVALID_ARG;
     }
     if (p->prescale && !lrq_aligned(p->prescale, 16)) return LRQ_ERR_INVALID_ARG;
@@ -66,7 +72,10 @@ static lrq_status check_act(const lrq_act_params* p, int K) {
 
 extern "C" size_t lrq_act_workspace_bytes(int M, int K, const lrq_act_params* p) {
     if (!p || M <= 0 || K <= 0) return 0;
-    return p->kind == LRQ_ROT_DENSE ? lrq_round_up((size_t)M * K * sizeof(float), 256) : 0;
+    const size_t rotated = lrq_round_up((size_t)M * K * sizeof(float), 256);
+    if (p->kind == LRQ_ROT_DENSE) return rotated;
+    if (p->kind == LRQ_ROT_DUAL) return rotated + lrq_round_up((size_t)M * K * 6, 256);   // + three bf16 panels
+    return 0;
 }
 
 extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long ldx, const lrq_act_params* p,
@@ -84,6 +93,20 @@ extern "C" lrq_status lrq_rotate_quantize_act(const void* X, int M, int K, long 
         // the rotation leaves each token's extremes in the scale / zero-point outputs (as integers); the
         // quantizer reads them and then writes the real values there
         st = lrq_launch_rotgemm(X, M, K, ldx, p->R_bf16, Yr, reinterpret_cast<int*>(a_scale), reinterpret_cast<int*>(a_zp), stream);
+        if (st != LRQ_OK) return st;
+        return lrq_launch_quantize_f32_ext(Yr, M, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
+    }
+    if (p->kind == LRQ_ROT_DUAL) {
+        const size_t need = lrq_act_workspace_bytes(M, K, p);
+        if (!workspace || workspace_bytes < need || !lrq_aligned(workspace, 256)) return LRQ_ERR_WORKSPACE;
+        float* Yr = static_cast<float*>(workspace);                       // u = x R1hat first, y later
+        void* V3 = static_cast<unsigned char*>(workspace) + lrq_round_up((size_t)M * K * sizeof(float), 256);
+        st = lrq_launch_bdiag_gemm(X, M, K, ldx, 1, p->R1_bf16, Yr, nullptr, nullptr, stream);
+        if (st != LRQ_OK) return st;
+        st = lrq_launch_dual_gather_split(Yr, M, K, p->perm, V3, stream);  // u P as three bf16 terms
+        if (st != LRQ_OK) return st;
+        st = lrq_launch_bdiag_gemm(V3, M, K, 3L * K, 3, p->R2_bf16, Yr, reinterpret_cast<int*>(a_scale),
+                                   reinterpret_cast<int*>(a_zp), stream);
         if (st != LRQ_OK) return st;
         return lrq_launch_quantize_f32_ext(Yr, M, K, p->a_bits, p->mode, a_codes, a_scale, a_zp, stream);
     }
@@ -114,10 +137,10 @@ extern "C" lrq_status lrq_rotate_quantize_act_static(const void* X, int M, int K
                                                      uint8_t* a_codes, float* a_scale, int32_t* a_zp,
                                                      void* cuda_stream) {
     if (!p) return LRQ_ERR_INVALID_ARG;
-    if (p->kind != LRQ_ROT_DENSE)                        // no scratch involved: the ordinary path, no workspace
+    if (p->kind != LRQ_ROT_DENSE && p->kind != LRQ_ROT_DUAL)   // no scratch involved: the ordinary path, no workspace
         return lrq_rotate_quantize_act(X, M, K, ldx, p, a_codes, a_scale, a_zp, nullptr, 0, cuda_stream);
     if (M <= 0 || K <= 0) return LRQ_ERR_INVALID_ARG;
-    if ((size_t)M * (size_t)K * sizeof(float) > (size_t)LRQ_STATIC_SCRATCH_BYTES) return LRQ_ERR_WORKSPACE;
+    if (lrq_act_workspace_bytes(M, K, p) > (size_t)LRQ_STATIC_SCRATCH_BYTES) return LRQ_ERR_WORKSPACE;
     void* scratch = static_scratch_address();
     if (!scratch) return LRQ_ERR_CUDA;
     return lrq_rotate_quantize_act(X, M, K, ldx, p, a_codes, a_scale, a_zp, scratch, LRQ_STATIC_SCRATCH_BYTES,
@@ -145,6 +168,15 @@ extern "C" lrq_status lrq_rotate_weights(const float* W, int N, int K, long ldw,
         return LRQ_ERR_INVALID_ARG;
     }
     return lrq_launch_rotate_weights(W, N, K, ldw, colmul, (int)kind, had_block, R_bf16, W_rot, ldo, (cudaStream_t)cuda_stream);
+}
+
+extern "C" lrq_status lrq_rotate_weights_dual(const float* W, int N, int K, long ldw, const float* colmul, int dual_block,
+                                              const void* R1_bf16, const int32_t* perm, const void* R2_bf16,
+                                              float* W_rot, long ldo, void* cuda_stream) {
+    if (!W || !W_rot || !R1_bf16 || !R2_bf16 || !perm || N <= 0 || K <= 0 || ldw < K || ldo < K) return LRQ_ERR_INVALID_ARG;
+    if (dual_block < 1 || K % dual_block) return LRQ_ERR_INVALID_ARG;
+    return lrq_launch_rotate_weights_dual(W, N, K, ldw, colmul, dual_block, R1_bf16, perm, R2_bf16, W_rot, ldo,
+                                          (cudaStream_t)cuda_stream);
 }
 
 extern "C" lrq_status lrq_layer_create(lrq_layer** out, int N, int K, int w_bits, int group_size,

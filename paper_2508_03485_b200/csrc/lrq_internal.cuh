@@ -68,6 +68,12 @@ lrq_status lrq_launch_rotq_blk(const void* X, int M, int K, long ldx, int B, int
 // maximum in ext_min[M] / ext_max[M] as order-preserving integers.
 lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y,
                               int* ext_min, int* ext_max, cudaStream_t st);
+// rotgemm.cu : Y[M,K] (fp32) = sum over the `parts` column panels of A[M, parts*K] (bf16) of panel . blockdiag(Rblk),
+// Rblk bf16 [K/128][128][128]; row extremes as above when ext_min / ext_max are given (both or neither).
+lrq_status lrq_launch_bdiag_gemm(const void* A, int M, int K, long lda, int parts, const void* Rblk, float* Y,
+                                 int* ext_min, int* ext_max, cudaStream_t st);
+// rotdual.cu : V3 bf16 [M,3K], panel p = p-th bf16 term of U[m, perm[i]] (the reordering between the two rotations)
+lrq_status lrq_launch_dual_gather_split(const float* U, int M, int K, const int32_t* perm, void* V3, cudaStream_t st);
 // rotq.cu : per-token quantization of fp32 rows whose extremes are already known (ext_min / ext_max alias the
 // scale / zero-point outputs: each row's extremes are read before its results are written).
 lrq_status lrq_launch_quantize_f32_ext(const float* Y, int M, int K, int a_bits, int mode, uint8_t* codes,
@@ -80,6 +86,8 @@ lrq_status lrq_launch_ars_metric(const void* X, int M, int K, long ldx, double t
 // wrot.cu : W diag(colmul) R in fp64, rounded to fp32 (Eq. 2, weight side)
 lrq_status lrq_launch_rotate_weights(const float* W, int N, int K, long ldw, const float* colmul, int kind,
                                      int had_block, const void* R, float* out, long ldo, cudaStream_t st);
+lrq_status lrq_launch_rotate_weights_dual(const float* W, int N, int K, long ldw, const float* colmul, int Bd, const void* R1,
+                                          const int32_t* perm, const void* R2, float* out, long ldo, cudaStream_t st);
 
 #ifdef __CUDACC__
 // Programmatic dependent launch.  Every hot kernel lets its successor in the stream start early (the successor's

@@ -11,6 +11,11 @@
 //   warps 2-5   epilogue: tcgen05.ld of the finished accumulator, fp32 stores
 // The accumulator is double-buffered in TMEM (2 x 256 columns).  Every wait is bounded; on expiry the
 // CTA records a code in the status word, waits (bounded) for its TMA loads in flight and unwinds.
+//
+// The same kernel, instantiated with 128-wide tiles, multiplies by a block-diagonal matrix of 128 x 128
+// blocks (the factors R1hat, R2hat of the dual transformation, Sec. 4.2): tile j of a token block only meets
+// block j, so its k-loop covers 128 input channels instead of K.  There the left operand may come in `parts`
+// column panels [M, parts*K] that are summed into one accumulator (the bf16 terms of an fp32 operand).
 #include "lrq_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tma_host.cuh"
@@ -19,12 +24,10 @@
 namespace {
 using namespace lrq_tc;
 
-constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int BM = 128, BK = 64;
 constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * BK * 2;          // 16 KB
 constexpr int B_CHUNK_BYTES = BK * 128;             // 8 KB: 64 k-rows of 64 output columns
-constexpr int B_STAGE_BYTES = (BN / 64) * B_CHUNK_BYTES;   // 32 KB
-constexpr int STAGE_TX_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, EPI_WARP0 = 2, NUM_EPI_WARPS = 4;
 constexpr int NUM_THREADS = (EPI_WARP0 + NUM_EPI_WARPS) * 32;   // 192
 constexpr int TMEM_COLS = 512;
@@ -38,13 +41,20 @@ struct __align__(16) Ctl {
     volatile int abort_flag;
 };
 constexpr int EPI_TILE_BYTES = 32 * 32 * 4;         // one epilogue warp's 32 x 32 fp32 chunk, for the row/column trade
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + sizeof(Ctl) + NUM_EPI_WARPS * EPI_TILE_BYTES;
+constexpr size_t smem_bytes(int bn) {
+    return 1024 + (size_t)STAGES * (A_STAGE_BYTES + (bn / 64) * B_CHUNK_BYTES) + sizeof(Ctl) + NUM_EPI_WARPS * EPI_TILE_BYTES;
+}
 
-constexpr uint32_t IDESC = umma_idesc_bf16(BM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
-
+// BN: tile width (256 dense; 128 = the diagonal block size when DIAG).  DIAG: R is block-diagonal, stored as its
+// blocks one after the other ([K/128][128][128], i.e. K rows of 128 columns); parts: column panels of the left operand.
+template <int BN, bool DIAG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmR,
-                  float* __restrict__ Y, int M, int K, int* __restrict__ ext_min, int* __restrict__ ext_max, int* status) {
+                  float* __restrict__ Y, int M, int K, int parts, int* __restrict__ ext_min, int* __restrict__ ext_max,
+                  int* status) {
+    constexpr int B_STAGE_BYTES = (BN / 64) * B_CHUNK_BYTES;   // 32 KB (16 KB for 128-wide tiles)
+    constexpr int STAGE_TX_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    constexpr uint32_t IDESC = umma_idesc_bf16(BM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     unsigned char* sA = base;
@@ -55,7 +65,9 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_m = (M + BM - 1) / BM, tiles_n = (K + BN - 1) / BN;
     const int num_tiles = tiles_m * tiles_n;
-    const int kblocks = (K + BK - 1) / BK;          // a ragged last k-block is zero-filled by TMA in both operands
+    // dense: the whole of K (a ragged last k-block is zero-filled by TMA in both operands);
+    // block-diagonal: the tile's own BN input channels, once per panel
+    const int kblocks = DIAG ? parts * (BN / BK) : (K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
@@ -85,10 +97,13 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                     if (!ok) break;
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     mbar_arrive_expect_tx(bar, STAGE_TX_BYTES);
-                    tma_load_2d(smem_u32(sA + s * A_STAGE_BYTES), &tmX, kb * BK, m0, bar);
+                    // k origin of this step in the left operand's columns and in R's rows
+                    const int kx = DIAG ? (kb / (BN / BK)) * K + n0 + (kb % (BN / BK)) * BK : kb * BK;
+                    const int kr = DIAG ? n0 + (kb % (BN / BK)) * BK : kb * BK;
+                    tma_load_2d(smem_u32(sA + s * A_STAGE_BYTES), &tmX, kx, m0, bar);
 #pragma unroll
                     for (int j = 0; j < BN / 64; ++j)
-                        tma_load_2d(smem_u32(sB + s * B_STAGE_BYTES + j * B_CHUNK_BYTES), &tmR, n0 + 64 * j, kb * BK, bar);
+                        tma_load_2d(smem_u32(sB + s * B_STAGE_BYTES + j * B_CHUNK_BYTES), &tmR, (DIAG ? 0 : n0) + 64 * j, kr, bar);
                 }
             }
             if (!ok) {
@@ -210,6 +225,32 @@ rotgemm_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 
 }  // namespace
 
+template <int BN, bool DIAG>
+static lrq_status launch_rotgemm(const CUtensorMap& tmX, const CUtensorMap& tmR, float* Y, int M, int K, int parts,
+                                 int* ext_min, int* ext_max, cudaStream_t st) {
+    int dev = 0, sms = 0;
+    if (lrq_current_device(&dev, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
+    {   // the shared-memory opt-in is a per-device function attribute: set once per device
+        static std::mutex mu;
+        static bool configured[LRQ_MAX_DEVICES] = {};
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[dev]) {
+            LRQ_CUDA_TRY(cudaFuncSetAttribute(rotgemm_tc_kernel<BN, DIAG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)smem_bytes(BN)));
+            configured[dev] = true;
+        }
+    }
+    const int tiles = ((M + BM - 1) / BM) * ((K + BN - 1) / BN);
+    if (ext_min) {
+        // identity elements of the integer min / max: bytes 0x7f.. (a huge float), 0x80.. (a hugely negative one)
+        LRQ_CUDA_TRY(cudaMemsetAsync(ext_min, 0x7f, (size_t)M * sizeof(int), st));
+        LRQ_CUDA_TRY(cudaMemsetAsync(ext_max, 0x80, (size_t)M * sizeof(int), st));
+    }
+    LRQ_CUDA_TRY(lrq_launch_pdl(rotgemm_tc_kernel<BN, DIAG>, dim3(tiles < sms ? tiles : sms), dim3(NUM_THREADS), smem_bytes(BN),
+                                st, tmX, tmR, Y, M, K, parts, ext_min, ext_max, lrq_status_word()));
+    return LRQ_OK;
+}
+
 lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void* R, float* Y,
                               int* ext_min, int* ext_max, cudaStream_t st) {
     // TMA needs 16-byte aligned bases and row pitches (K and ldx multiples of 8 elements); the C ABI has already
@@ -219,22 +260,18 @@ lrq_status lrq_launch_rotgemm(const void* X, int M, int K, long ldx, const void*
     CUtensorMap tmX, tmR;
     if (!lrq_tma::make_map_2d(&tmX, X, 2, (uint64_t)M, (uint64_t)K, (uint64_t)ldx, BK, BM, true)) return LRQ_ERR_CUDA;
     if (!lrq_tma::make_map_2d(&tmR, R, 2, (uint64_t)K, (uint64_t)K, (uint64_t)K, 64, BK, true)) return LRQ_ERR_CUDA;
-    int dev = 0, sms = 0;
-    if (lrq_current_device(&dev, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
-    {   // the shared-memory opt-in is a per-device function attribute: set once per device
-        static std::mutex mu;
-        static bool configured[LRQ_MAX_DEVICES] = {};
-        std::lock_guard<std::mutex> lock(mu);
-        if (!configured[dev]) {
-            LRQ_CUDA_TRY(cudaFuncSetAttribute(rotgemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-            configured[dev] = true;
-        }
-    }
-    const int tiles = ((M + BM - 1) / BM) * ((K + BN - 1) / BN);
-    // identity elements of the integer min / max: bytes 0x7f.. (a huge float), 0x80.. (a hugely negative one)
-    LRQ_CUDA_TRY(cudaMemsetAsync(ext_min, 0x7f, (size_t)M * sizeof(int), st));
-    LRQ_CUDA_TRY(cudaMemsetAsync(ext_max, 0x80, (size_t)M * sizeof(int), st));
-    LRQ_CUDA_TRY(lrq_launch_pdl(rotgemm_tc_kernel, dim3(tiles < sms ? tiles : sms), dim3(NUM_THREADS), SMEM_BYTES, st, tmX, tmR,
-                                Y, M, K, ext_min, ext_max, lrq_status_word()));
-    return LRQ_OK;
+    return launch_rotgemm<256, false>(tmX, tmR, Y, M, K, 1, ext_min, ext_max, st);
+}
+
+// Y[M,K] (fp32) = sum over panels p of A[:, pK .. pK+K) . blockdiag(Rblk), Rblk bf16 [K/128][128][128].
+// ext_min / ext_max may both be null (no per-row extremes wanted).
+lrq_status lrq_launch_bdiag_gemm(const void* A, int M, int K, long lda, int parts, const void* Rblk, float* Y,
+                                 int* ext_min, int* ext_max, cudaStream_t st) {
+    if ((K % 128) || (lda % 8) || lda < (long)parts * K || parts < 1 || !lrq_aligned(A, 16) || !lrq_aligned(Rblk, 16) ||
+        !lrq_aligned(Y, 16) || (ext_min == nullptr) != (ext_max == nullptr))
+        return LRQ_ERR_INVALID_ARG;
+    CUtensorMap tmA, tmR;
+    if (!lrq_tma::make_map_2d(&tmA, A, 2, (uint64_t)M, (uint64_t)parts * K, (uint64_t)lda, BK, BM, true)) return LRQ_ERR_CUDA;
+    if (!lrq_tma::make_map_2d(&tmR, Rblk, 2, (uint64_t)K, 128, 128, 64, BK, true)) return LRQ_ERR_CUDA;
+    return launch_rotgemm<128, true>(tmA, tmR, Y, M, K, parts, ext_min, ext_max, st);
 }

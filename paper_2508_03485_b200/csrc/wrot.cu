@@ -5,7 +5,8 @@
 // Offline step.  Hadamard: one CTA per weight row, the row in shared memory as fp64, log2(B) butterfly
 // stages with a CTA barrier between them.  Dense: an fp64 matrix product on the CUDA cores, 64 x 64
 // output tiles, 4 x 4 accumulators per thread; R is the layer's stored bf16 matrix (exact in fp64), so
-// both sides of Eq. 2 use the same R.
+// both sides of Eq. 2 use the same R.  Dual transformation (R = R1hat P R2hat, Sec. 4.2): one CTA per row, the
+// row in shared memory as fp64, block-diagonal product, gather through the index map, second product.
 #include "lrq_internal.cuh"
 
 #include <cuda_bf16.h>
@@ -89,6 +90,43 @@ wrot_dense_kernel(const float* __restrict__ W, int N, int K, long ldw, const flo
     }
 }
 
+// out[n] = ((w[n] * colmul) . blockdiag(R1)) gathered through perm, then . blockdiag(R2); blocks of Bd x Bd, row-major
+__global__ void __launch_bounds__(256)
+wrot_dual_kernel(const float* __restrict__ W, int N, int K, long ldw, const float* __restrict__ colmul, int Bd,
+                 const __nv_bfloat16* __restrict__ R1, const int32_t* __restrict__ perm, const __nv_bfloat16* __restrict__ R2,
+                 float* __restrict__ out, long ldo) {
+    extern __shared__ double rows2[];              // a[K], b[K]
+    double* a = rows2;
+    double* b = rows2 + K;
+    const int n = blockIdx.x, tid = threadIdx.x;
+    const float* w = W + (size_t)n * ldw;
+    for (int k = tid; k < K; k += 256) a[k] = (double)w[k] * (colmul ? (double)colmul[k] : 1.0);
+    __syncthreads();
+    for (int c = tid; c < K; c += 256) {           // b = a . blockdiag(R1)
+        const int j = c / Bd, i = c - j * Bd;
+        const __nv_bfloat16* r = R1 + (size_t)j * Bd * Bd + i;
+        const double* x = a + j * Bd;
+        double acc = 0.0;
+        for (int l = 0; l < Bd; ++l) acc = fma(x[l], (double)__bfloat162float(r[(size_t)l * Bd]), acc);
+        b[c] = acc;
+    }
+    __syncthreads();
+    for (int c = tid; c < K; c += 256) {           // a = b . P
+        const int p = perm[c];
+        a[c] = (uint32_t)p < (uint32_t)K ? b[p] : b[0];
+    }
+    __syncthreads();
+    float* o = out + (size_t)n * ldo;
+    for (int c = tid; c < K; c += 256) {           // out = a . blockdiag(R2)
+        const int j = c / Bd, i = c - j * Bd;
+        const __nv_bfloat16* r = R2 + (size_t)j * Bd * Bd + i;
+        const double* x = a + j * Bd;
+        double acc = 0.0;
+        for (int l = 0; l < Bd; ++l) acc = fma(x[l], (double)__bfloat162float(r[(size_t)l * Bd]), acc);
+        o[c] = (float)acc;
+    }
+}
+
 __global__ void wrot_scale_kernel(const float* __restrict__ W, int N, int K, long ldw, const float* __restrict__ colmul,
                                   float* __restrict__ out, long ldo) {
     const size_t total = (size_t)N * K;
@@ -118,6 +156,18 @@ lrq_status lrq_launch_rotate_weights(const float* W, int N, int K, long ldw, con
         const int blocks = (int)((total + 255) / 256 < 4096 ? (total + 255) / 256 : 4096);
         wrot_scale_kernel<<<blocks, 256, 0, st>>>(W, N, K, ldw, colmul, out, ldo);
     }
+    LRQ_CUDA_TRY(cudaGetLastError());
+    return LRQ_OK;
+}
+
+lrq_status lrq_launch_rotate_weights_dual(const float* W, int N, int K, long ldw, const float* colmul, int Bd, const void* R1,
+                                          const int32_t* perm, const void* R2, float* out, long ldo, cudaStream_t st) {
+    const size_t smem = (size_t)K * 2 * sizeof(double);
+    if (smem > 200 * 1024) return LRQ_ERR_UNSUPPORTED;
+    if (smem > 40 * 1024)
+        LRQ_CUDA_TRY(cudaFuncSetAttribute(wrot_dual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    wrot_dual_kernel<<<N, 256, smem, st>>>(W, N, K, ldw, colmul, Bd, static_cast<const __nv_bfloat16*>(R1), perm,
+                                           static_cast<const __nv_bfloat16*>(R2), out, ldo);
     LRQ_CUDA_TRY(cudaGetLastError());
     return LRQ_OK;
 }

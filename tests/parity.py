@@ -29,15 +29,20 @@ boundary_tol, in code steps, for an element with t = y/s of a token with zero-po
         round toward zero: each loses up to one ulp (2u) of the running sum, half of that on average.  The part
         common to a token's elements (a uniform shrink) cancels in y/s; what is left is bounded here by
         (K/32) * u * rms(y), half an ulp per chained add (measured worst case: 0.45 of it at K = 3072);
+      dual (two block-diagonal products of Bd-wide blocks, the second over the three bf16 terms of the first one's
+        fp32 result): Bd/16 chained adds, then 3 Bd/16 of them, counted as for the dense product: (4 Bd / 32) * u *
+        rms(y) (the second rotation is orthogonal, so the first product's error keeps its size on the way through;
+        what the three-term split drops, 2^-25 of each element, is below one rounding);
       none: y is the bf16 input, exact.
-    tol = u * (4 * (|t| + |z| + 1) + g * rms(y)/s),  g = sqrt(log2 B), K/32 or 0
+    tol = u * (4 * (|t| + |z| + 1) + g * rms(y)/s),  g = sqrt(log2 B), K/32, Bd/8 or 0
     (the first term is a worst-case bound; measured on the five workloads, differing elements sit within 0.2 tol).
 Scale tolerance: s is (max - min) / (2^b - 1) of fp32 extremes, evaluated in fp64 and rounded to fp32 once:
     Hadamard / none: 5e-7 relative = 8 u (the fp32 rounding of s itself is u; the extremes' rotation error is a few u
     of their magnitude; measured 1e-7);
     dense: the extremes carry the tensor-core accumulation error; if every one of the K/16 accumulations
     truncated in the same direction the relative error would reach (K/16) * 2^-23, which is the bound used
-    (2.3e-5 at K = 3072; measured 2.7e-6 at K = 1536); never below 5e-7.
+    (2.3e-5 at K = 3072; measured 2.7e-6 at K = 1536); never below 5e-7;
+    dual: the same with the 4 Bd / 16 chained accumulations of its two products (3.8e-6 for Bd = 128).
 """
 from __future__ import annotations
 
@@ -86,13 +91,19 @@ def rotation_gain(rot: str, K: int, had_block: int = 0) -> float:
         return float(np.sqrt(max(1.0, np.log2(max(had_block, 2)))))
     if rot == "dense":
         return float(K / 32.0)
+    if rot == "dual":                      # had_block carries Bd
+        return float(had_block / 8.0)
     if rot == "none":
         return 0.0
     raise ValueError(rot)
 
 
-def scale_rtol(rot: str, K: int) -> float:
-    return max(5e-7, (K / 16.0) * 2.0 ** -23) if rot == "dense" else 5e-7
+def scale_rtol(rot: str, K: int, had_block: int = 0) -> float:
+    if rot == "dense":
+        return max(5e-7, (K / 16.0) * 2.0 ** -23)
+    if rot == "dual":                      # had_block carries Bd
+        return max(5e-7, (4 * had_block / 16.0) * 2.0 ** -23)
+    return 5e-7
 
 
 @dataclass
@@ -121,7 +132,7 @@ def check_act(gpu_q, gpu_s, gpu_z, orc_q, orc_s, orc_z, orc_y, rot, had_block=0,
     assert gpu_q.shape == orc_q.shape == orc_y.shape
     gz, oz = np.asarray(gpu_z, dtype=np.int64), np.asarray(orc_z, dtype=np.int64)
     gs, os_ = np.asarray(gpu_s, dtype=np.float64), np.asarray(orc_s, dtype=np.float64)
-    rtol = scale_rtol(rot, K)
+    rtol = scale_rtol(rot, K, had_block)
     rel_s = np.abs(gs - os_) / os_
     assert (rel_s <= rtol).all(), f"{what}: scales differ by {rel_s.max():.2e} relative (limit {rtol:.1e})"
 
@@ -233,20 +244,36 @@ def check_tlq(orc, W: np.ndarray, tl, bits: int, group: int, rows=None, what="",
     return T
 
 
+def dual_to_device(P, factors):
+    """(Bd, R1 bits, perm, R2 bits) of LayerSpec.dual_factors -> the binding's DualRotation on the device."""
+    Bd, R1, perm, R2 = factors
+    return P.DualRotation(Bd, bf16_to_device(R1), torch.from_numpy(np.ascontiguousarray(perm, dtype=np.int32)).cuda(),
+                          bf16_to_device(R2))
+
+
+def dual_to_f64(factors):
+    """The same factors as the oracle takes them."""
+    Bd, R1, perm, R2 = factors
+    return Bd, bf16_bits_to_f64(R1), perm, bf16_bits_to_f64(R2)
+
+
 def gpu_layer(spec: LayerSpec, W: np.ndarray, P, code_layout: int = 0):
     """Quantize weights on the GPU and build the layer handle.  Returns (QLayer, TLQWeights)."""
     g = default_clip_grid()
     Wd = torch.from_numpy(W).cuda()
     tl = P.lrq_tlq_quantize_weights(Wd, spec.w_bits, spec.group, 7, g, g, code_layout=code_layout)
-    R = None
+    R = dual = None
     if spec.rot == "dense":
         R = bf16_to_device(spec.rotation_bf16())
-    kind = P.ROT_DENSE if spec.rot == "dense" else P.ROT_HADAMARD
-    return P.QLayer(tl, spec.N, spec.K, kind, spec.a_bits, spec.had_block, R), tl
+    if spec.rot == "dual":
+        dual = dual_to_device(P, spec.dual_factors())
+    kind = {"dense": P.ROT_DENSE, "dual": P.ROT_DUAL, "hadamard": P.ROT_HADAMARD}[spec.rot]
+    return P.QLayer(tl, spec.N, spec.K, kind, spec.a_bits, spec.had_block, R, dual=dual), tl
 
 
 def oracle_layer_rows(orc, spec: LayerSpec, Xbits_rows: np.ndarray, T, R_bits=None):
     """The oracle's whole layer on the given token rows: (Y, codes, s, z, rotated values)."""
     X = bf16_bits_to_f64(Xbits_rows)
     R = None if R_bits is None else bf16_bits_to_f64(R_bits)
-    return orc.qlinear(X, T, spec.a_bits, spec.rot, spec.had_block, R, return_rotated=True)
+    dual = dual_to_f64(spec.dual_factors()) if spec.rot == "dual" else None
+    return orc.qlinear(X, T, spec.a_bits, spec.rot, spec.had_block, R, return_rotated=True, dual=dual)

@@ -1,0 +1,165 @@
+"""The dual transformation kept in its factors (Sec. 4.2: y = x . R1hat . P . R2hat) on the GPU against the oracle:
+activation codes, the weight side of Eq. 2, a whole layer, and the shapes of the dense layers of the FLUX- and
+PixArt-like workloads, with the time of the dense-matrix path beside it."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import parity as PU
+from lrq_workloads import (LayerSpec, bf16_bits_to_f64, config_layers, default_clip_grid, f32_to_bf16_bits,
+                           make_activations, make_weights)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2508_03485_b200 as P
+    P.load_library()
+    return P
+
+
+def _spec(M, K, N=128, a_bits=8, w_bits=4, seed=71, n_salient=16):
+    return LayerSpec("dual", seed, M, K, N, w_bits, a_bits, 0, "dual", 128, n_salient=n_salient, salient_x=100.0)
+
+
+def _codes_against_oracle(P, orc, spec, xb, what):
+    f = spec.dual_factors()
+    dual = PU.dual_to_device(P, f)
+    q, s, z = P.lrq_rotate_quantize_act(PU.bf16_to_device(xb), P.ROT_DUAL, spec.a_bits, dual=dual)
+    torch.cuda.synchronize()
+    assert P.lrq_device_status() == 0
+    Yr = orc.rotate_dual(bf16_bits_to_f64(xb), *PU.dual_to_f64(f))
+    oq, os_, oz = orc.quantize_act(Yr, spec.a_bits)
+    return PU.check_act(PU.act_codes_to_numpy(q, spec.a_bits), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, Yr,
+                        "dual", 128, what)
+
+
+@pytest.mark.parametrize("M,K,a_bits", [(70, 128, 8), (70, 256, 4), (130, 1152, 8), (33, 1536, 4), (300, 3072, 4),
+                                        (1, 384, 8)])
+def test_rotate_quantize_dual(P, orc, M, K, a_bits):
+    spec = _spec(M, K, a_bits=a_bits)
+    _codes_against_oracle(P, orc, spec, spec.activations(), f"dual {M}x{K}")
+
+
+def test_dual_with_identity_factors_is_the_reordering(P, orc):
+    # R1 = R2 = I: the rotated values are the bf16 inputs themselves in the new order, so the codes must be the
+    # codes of the permuted input (exact ties aside, as for any unrotated bf16 input)
+    M, K = 40, 512
+    spec = _spec(M, K)
+    xb = spec.activations()
+    Bd, _, perm, _ = spec.dual_factors()
+    eye = f32_to_bf16_bits(np.broadcast_to(np.eye(Bd, dtype=np.float32), (K // Bd, Bd, Bd)).copy())
+    dual = PU.dual_to_device(P, (Bd, eye, perm, eye))
+    q, s, z = P.lrq_rotate_quantize_act(PU.bf16_to_device(xb), P.ROT_DUAL, 8, dual=dual)
+    Yn = bf16_bits_to_f64(xb)[:, perm]
+    oq, os_, oz = orc.quantize_act(Yn, 8)
+    PU.check_act(PU.act_codes_to_numpy(q, 8), s.cpu().numpy(), z.cpu().numpy(), oq, os_, oz, Yn, "none", 0, "identity dual")
+
+
+def test_bad_index_map_entry_is_recorded_not_followed(P):
+    spec = _spec(8, 256)
+    Bd, R1, perm, R2 = spec.dual_factors()
+    bad = perm.copy()
+    bad[5] = 256                                                  # one past the end
+    dual = PU.dual_to_device(P, (Bd, R1, bad, R2))
+    P.lrq_rotate_quantize_act(PU.bf16_to_device(spec.activations()), P.ROT_DUAL, 8, dual=dual)
+    torch.cuda.synchronize()
+    assert P.lrq_device_status() == 31
+    assert P.lrq_device_status() == 0
+
+
+def test_dual_argument_checks(P):
+    spec = _spec(8, 256)
+    X = PU.bf16_to_device(spec.activations())
+    Bd, R1, perm, R2 = spec.dual_factors()
+    d64 = P.DualRotation(64, PU.bf16_to_device(R1).reshape(4, 64, 128)[:, :, :64].contiguous(),
+                         torch.from_numpy(perm).cuda(), PU.bf16_to_device(R2).reshape(4, 64, 128)[:, :, :64].contiguous())
+    with pytest.raises(P.LrqError) as e:                          # only 128-wide blocks are built
+        P.lrq_rotate_quantize_act(X, P.ROT_DUAL, 8, dual=d64)
+    assert e.value.code == 2
+    with pytest.raises(P.LrqError) as e:                          # factors missing
+        P.lrq_rotate_quantize_act(X, P.ROT_DUAL, 8)
+    assert e.value.code == 1
+
+
+@pytest.mark.parametrize("N,K,smooth", [(37, 1152, True), (9, 256, False), (4, 12288, False)])
+def test_rotate_weights_dual(P, orc, N, K, smooth):
+    spec = _spec(8, K, N)
+    f = spec.dual_factors()
+    W = make_weights(33, N, K)
+    c = np.random.default_rng(K).uniform(0.3, 3.0, K).astype(np.float32) if smooth else None
+    out = P.lrq_rotate_weights_dual(torch.from_numpy(W).cuda(), PU.dual_to_device(P, f),
+                                    None if c is None else torch.from_numpy(c).cuda())
+    ref = orc.rotate_weights(W.astype(np.float64), None if c is None else c.astype(np.float64), "dual",
+                             dual=PU.dual_to_f64(f))
+    got = out.cpu().numpy()
+    ref32 = ref.astype(np.float32)
+    ulp = np.spacing(np.abs(ref32)).astype(np.float64)
+    assert (np.abs(got.astype(np.float64) - ref) <= 0.5 * ulp + 1e-12 * np.abs(ref).max()).all()
+    assert (got != ref32).mean() < 1e-3
+
+
+@pytest.mark.parametrize("M,K,N,w_bits,a_bits", [(200, 1152, 264, 4, 8), (130, 1536, 136, 3, 4)])
+def test_dual_layer_end_to_end(P, orc, M, K, N, w_bits, a_bits):
+    # weights through lrq_rotate_weights_dual, so that both sides of Eq. 2 use the same factors; then the whole layer
+    spec = _spec(M, K, N, a_bits, w_bits, seed=83)
+    f = spec.dual_factors()
+    W = spec.weights()
+    Wr = P.lrq_rotate_weights_dual(torch.from_numpy(W).cuda(), PU.dual_to_device(P, f)).cpu().numpy()
+    layer, tl = PU.gpu_layer(spec, Wr, P)
+    T = PU.check_tlq(orc, Wr, tl, w_bits, 0, what="dual tlq")
+    xb = spec.activations()
+    Yo, oq, os_, oz, Yr = PU.oracle_layer_rows(orc, spec, xb, T)
+    X = PU.bf16_to_device(xb)
+    q, s, z = P.lrq_rotate_quantize_act(X, P.ROT_DUAL, a_bits, dual=layer.dual)
+    gq, gz = PU.act_codes_to_numpy(q, a_bits), z.cpu().numpy()
+    act = PU.check_act(gq, s.cpu().numpy(), gz, oq, os_, oz, Yr, "dual", 128, "dual layer codes")
+    Y = P.lrq_qlinear(layer, X, P.F32)
+    PU.check_layer_out(orc, T, Y.cpu().numpy(), gq, gz, Yo, os_, act, "dual layer")
+    # Eq. 2: the rotated, quantized layer estimates the plain product X W^T
+    plain = bf16_bits_to_f64(xb) @ W.astype(np.float64).T
+    err = np.linalg.norm(Y.cpu().numpy() - plain) / np.linalg.norm(plain)
+    err_oracle = np.linalg.norm(Yo - plain) / np.linalg.norm(plain)
+    # the quantizers' error (the oracle's own), far from what mismatched sides of Eq. 2 would give (order one)
+    assert err_oracle < (0.35 if a_bits == 8 else 0.75) and abs(err - err_oracle) < 0.01, (err, err_oracle)
+    assert P.lrq_device_status() == 0
+
+
+def _time_ms(fn, reps=10):
+    fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+@pytest.mark.parametrize("cfg,name", [(3, "qkv"), (2, "proj"), (2, "fc1")])
+def test_dual_at_workload_shapes(P, orc, cfg, name):
+    # the dense layers of the FLUX- and PixArt-like workloads with their rotation kept in factors: codes of every
+    # token against the oracle, and the two paths' rotate+quantize times side by side (printed, not asserted)
+    base = next(s for s in config_layers(cfg) if s.name == name)
+    spec = dataclasses.replace(base, rot="dual", had_block=128)
+    xb = spec.activations()
+    r = _codes_against_oracle(P, orc, spec, xb, f"cfg{cfg} {name} dual")
+    X = PU.bf16_to_device(xb)
+    dual = PU.dual_to_device(P, spec.dual_factors())
+    R = PU.bf16_to_device(base.rotation_bf16())
+    lib = P.load_library()
+    ws = torch.empty(10 * spec.M * spec.K + 4096, dtype=torch.uint8, device="cuda")
+    out = (torch.empty((spec.M, spec.K * spec.a_bits // 8), dtype=torch.uint8, device="cuda"),
+           torch.empty(spec.M, dtype=torch.float32, device="cuda"), torch.empty(spec.M, dtype=torch.int32, device="cuda"))
+    t_dual = _time_ms(lambda: P.lrq_rotate_quantize_act(X, P.ROT_DUAL, spec.a_bits, dual=dual, workspace=ws, out=out))
+    t_dense = _time_ms(lambda: P.lrq_rotate_quantize_act(X, P.ROT_DENSE, spec.a_bits, R=R, workspace=ws, out=out))
+    print(f"\ncfg{cfg} {name} M={spec.M} K={spec.K} A{spec.a_bits}: rotate+quantize dual {t_dual * 1e3:.1f} us, "
+          f"dense {t_dense * 1e3:.1f} us; flips {r.flip_fraction:.2e}, worst boundary {r.worst_boundary:.2f}, "
+          f"worst scale {r.worst_scale:.2f}")
+    assert P.lrq_device_status() == 0

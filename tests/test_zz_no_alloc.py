@@ -41,6 +41,7 @@ def test_static_scratch_matches_workspace_path_twice(P):
         out = (torch.empty((M, K * a_bits // 8), dtype=torch.uint8, device="cuda"),
                torch.empty((M,), dtype=torch.float32, device="cuda"),
                torch.empty((M,), dtype=torch.int32, device="cuda"))
+        got = None                                                             # drop the previous round's buffers now
         torch.cuda.synchronize()
         held, reserved, free = torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), _free_bytes()
         got = P.lrq_rotate_quantize_act_static(X, P.ROT_DENSE, a_bits, R=R, out=out)
@@ -72,3 +73,20 @@ def test_static_scratch_other_kinds_and_limit(P):
     out = P.lrq_rotate_quantize_act_static(Xb[:-1], P.ROT_DENSE, 8, R=Rb)   # exactly at the limit
     torch.cuda.synchronize()
     assert int(out[2].abs().max()) == 0
+
+
+def test_static_scratch_serves_the_dual_transformation(P):
+    # kind DUAL needs 10 bytes of scratch per element (fp32 rotated values and three bf16 panels)
+    from lrq_workloads import LayerSpec
+    spec = LayerSpec("dual", 17, 300, 384, 8, 4, 8, 0, "dual", 128, n_salient=8)
+    dual = PU.dual_to_device(P, spec.dual_factors())
+    X = PU.bf16_to_device(spec.activations())
+    ref = P.lrq_rotate_quantize_act(X, P.ROT_DUAL, 8, dual=dual)
+    got = P.lrq_rotate_quantize_act_static(X, P.ROT_DUAL, 8, dual=dual)
+    torch.cuda.synchronize()
+    for g, r in zip(got, ref):
+        assert torch.equal(g, r)
+    M = P.lrq_static_scratch_bytes() // (10 * 384) + 2
+    with pytest.raises(P.LrqError) as e:
+        P.lrq_rotate_quantize_act_static(torch.zeros((M, 384), dtype=torch.bfloat16, device="cuda"), P.ROT_DUAL, 8, dual=dual)
+    assert e.value.code == 3
