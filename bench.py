@@ -47,6 +47,10 @@ NCU_TRAFFIC_BYTES = {
     "rotgemm cfg3 qkv": 51.51e6 + 19.17e6 + 56.67e6 + 0.25e6,
 }
 
+# sm__pipe_tensor_cycles_active (% of elapsed cycles) of the same captures: the tensor pipe's own view of the
+# contraction, beside the fraction of the measured matmul peak that `frac` reports
+NCU_TENSOR_PIPE_PCT = {"qgemm cfg4 b0.fc1": 46.0, "qgemm cfg3 fc1": 54.0}
+
 METRIC = "qlinear_tflops"
 UNIT = "TFLOP/s"
 ORACLE_SAMPLE_TOKENS = 128
@@ -310,6 +314,7 @@ def kernel_objects(P, torch, W, timed, peaks, out_name, gemm_impl=0, want_dense=
                            "achieved": gemm_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": gemm_tf / peaks["bf16_tflops"],
                            "traffic": NCU_TRAFFIC_BYTES.get(f"qgemm cfg{cfg} {s.name}") if out_name == "f32" else None,
                            "traffic_unit": "bytes per launch (ncu dram read + write)", "algorithmic_flops": 2.0 * s.M * s.N * s.K,
+                           "tensor_pipe_active_pct_ncu": NCU_TENSOR_PIPE_PCT.get(f"qgemm cfg{cfg} {s.name}") if out_name == "f32" else None,
                            "peak_source": peaks["source"] + " burst bf16 (kernel timed alone)", "ms": gemm_ms}
     del q, sc, zp
     had = [i for i in range(len(specs)) if specs[i].rot == "hadamard"]
@@ -343,6 +348,20 @@ def kernel_objects(P, torch, W, timed, peaks, out_name, gemm_impl=0, want_dense=
                                     "peak_source": peaks["source"] + " burst bf16 (both kernels of the dense path timed together)",
                                     "ms": d_ms}
         del rq, wsd
+        if sd.K % 128 == 0:
+            # the same layer with its rotation kept in the factors of the dual transformation (seeded block rotations
+            # around a staggered reordering): rotate+quantize of all tokens, beside the dense-matrix path above
+            Bd, R1, perm, R2 = sd.dual_factors()
+            dual = P.DualRotation(Bd, bf16_tensor(torch, R1).to(W.dev), torch.from_numpy(perm).to(W.dev),
+                                  bf16_tensor(torch, R2).to(W.dev))
+            wsu = torch.empty(10 * sd.M * sd.K + 4096, dtype=torch.uint8, device=W.dev)
+            rq = P.lrq_rotate_quantize_act(W.Xs[d], P.ROT_DUAL, sd.a_bits, dual=dual, workspace=wsu)
+            u_ms = float(np.mean(timed(lambda: P.lrq_rotate_quantize_act(W.Xs[d], P.ROT_DUAL, sd.a_bits, dual=dual, workspace=wsu,
+                                                                         stream=stream, out=rq), 20)))
+            out["rotdual"] = {"kernel": f"dual rotation (two block-diagonal products, reordering between) + quantizer cfg{cfg} {sd.name} "
+                                        f"{sd.M}x{sd.K} Bd{Bd} A{sd.a_bits}", "ms": u_ms, "dense_path_ms": d_ms,
+                              "algorithmic_flops": 2.0 * sd.M * sd.K * Bd * 4}
+            del rq, wsu, dual
     return out
 
 
@@ -510,8 +529,9 @@ def run_cuda(args):
                              "tokens_per_s": ORACLE_SAMPLE_TOKENS / osec},
             "tlq_weight_quantization": {"weights_per_s": W.n_weights / (W.tlq_ms * 1e-3), "ms": W.tlq_ms},
         }
-        if "roofline_rotdense" in objs:
-            line["roofline_rotdense"] = objs["roofline_rotdense"]
+        for k in ("roofline_rotdense", "rotdual"):
+            if k in objs:
+                line[k] = objs[k]
         line.update(extra)
         print(json.dumps(line))
     if world > 1:
