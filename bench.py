@@ -422,33 +422,40 @@ def run_cuda(args):
     h2d = sum(h.numel() * 2 for h, _ in uniq_x.values())
     d2h = sum(y.numel() * y.element_size() for y in uniq_y.values())
 
-    # One lrq_qlinear call per layer on the compute stream; uploads run on a second stream and read-backs on a third,
-    # so a layer's upload and the previous layer's read-back overlap its kernels.  A shared activation buffer is
-    # uploaded once, before its first reader; an output buffer is read back after its last writer.
+    # One lrq_qlinear call per layer (and token chunk) on the compute stream; uploads run on a second stream and
+    # read-backs on a third.  An output buffer is read back after its last writer.
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
     first_reader, last_writer = {}, {}
     for i, (x, y) in enumerate(zip(Xs, Ys)):
         first_reader.setdefault(id(x), i)
         last_writer[id(y)] = i
 
+    # A large batch goes through in token chunks (tokens are independent through the whole path): chunk c's outputs
+    # travel back to the host while chunk c + 1 is computed, and its activations arrive while chunk c - 1 is computed.
+    # The chunks shrink towards the end: only the last chunk's read-back is left over when the kernels are done.
+    m_all = Xs[0].shape[0]
+    chunked = m_all >= 16384 and m_all % 16 == 0 and all(x.shape[0] == m_all for x in Xs)
+    bounds = [0, m_all * 6 // 16, m_all * 11 // 16, m_all * 14 // 16, m_all] if chunked else [0, m_all]
+    nch = len(bounds) - 1
+
     def e2e_step():
-        s_in.wait_stream(stream)
-        uploaded = {}
-        with torch.cuda.stream(s_in):
-            for h, d in uniq_x.values():
-                d.copy_(h, non_blocking=True)
-                uploaded[id(d)] = torch.cuda.Event()
-                uploaded[id(d)].record(s_in)
-        for i, (L, x, y) in enumerate(zip(layers, Xs, Ys)):
-            if first_reader[id(x)] == i:
-                stream.wait_event(uploaded[id(x)])
-            P.lrq_qlinear(L, x, ydt, out=y, workspace=W.ws, stream=stream)
-            if last_writer[id(y)] == i:
-                done = torch.cuda.Event()
-                done.record(stream)
-                s_out.wait_event(done)
-                with torch.cuda.stream(s_out):
-                    y_host[id(y)].copy_(y, non_blocking=True)
+        s_in.wait_stream(stream)          # the previous step's kernels have read the activation buffers
+        for c in range(nch):
+            rows = slice(bounds[c], bounds[c + 1])
+            with torch.cuda.stream(s_in):
+                for h, d in uniq_x.values():
+                    d[rows].copy_(h[rows], non_blocking=True)
+                uploaded = torch.cuda.Event()
+                uploaded.record(s_in)
+            stream.wait_event(uploaded)
+            for i, (L, x, y) in enumerate(zip(layers, Xs, Ys)):
+                P.lrq_qlinear(L, x[rows], ydt, out=y[rows], workspace=W.ws, stream=stream)
+                if last_writer[id(y)] == i:
+                    done = torch.cuda.Event()
+                    done.record(stream)
+                    s_out.wait_event(done)
+                    with torch.cuda.stream(s_out):
+                        y_host[id(y)][rows].copy_(y[rows], non_blocking=True)
         stream.wait_stream(s_out)
 
     for _ in range(2):
@@ -521,7 +528,7 @@ def run_cuda(args):
                                             "timed alone are compared with the burst figure"},
             "tokens_per_s": world * tokens / (ms_step * 1e-3),
             "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": e2e_ms, "launch": "one lrq_qlinear call per layer; copies on two side streams"},
+                    "ms_per_step": e2e_ms, "launch": f"one lrq_qlinear call per layer and token chunk ({nch} chunk(s)); copies on two side streams"},
             "gpu_launches": args.steps * W.launches_per_step(),
             "clocks": clocks, "roofline": objs["roofline"], "roofline_rotq": objs.get("roofline_rotq"),
             "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
