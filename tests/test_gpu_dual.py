@@ -163,3 +163,23 @@ def test_dual_at_workload_shapes(P, orc, cfg, name):
           f"dense {t_dense * 1e3:.1f} us; flips {r.flip_fraction:.2e}, worst boundary {r.worst_boundary:.2f}, "
           f"worst scale {r.worst_scale:.2f}")
     assert P.lrq_device_status() == 0
+
+
+def test_stack_with_a_dual_layer_matches_single_calls(P):
+    specs = [LayerSpec("a", 91, 64, 256, 72, 4, 8, 0, "hadamard", 128),
+             LayerSpec("b", 92, 130, 384, 136, 4, 8, 0, "dual", 128, n_salient=8),
+             LayerSpec("c", 93, 33, 128, 136, 3, 4, 0, "dense", 0)]
+    layers, Xs, Ys, refs = [], [], [], []
+    for sp in specs:
+        layer, _ = PU.gpu_layer(sp, sp.weights(), P)
+        X = PU.bf16_to_device(sp.activations())
+        layers.append(layer); Xs.append(X)
+        refs.append(P.lrq_qlinear(layer, X, P.F32))
+        Ys.append(torch.zeros_like(refs[-1]))
+    plan = P.StackPlan(layers, Xs, Ys, P.F32)
+    assert plan.need >= 10 * 130 * 384                            # the dual layer's scratch sizes the shared workspace
+    P.lrq_qlinear_stack(plan)
+    torch.cuda.synchronize()
+    for y, r in zip(Ys, refs):
+        assert torch.equal(y, r)
+    assert P.lrq_device_status() == 0
