@@ -40,7 +40,7 @@ def _codes_against_oracle(P, orc, spec, xb, what):
 
 
 @pytest.mark.parametrize("M,K,a_bits", [(70, 128, 8), (70, 256, 4), (130, 1152, 8), (33, 1536, 4), (300, 3072, 4),
-                                        (1, 384, 8)])
+                                        (1, 384, 8), (40, 12288, 4), (130, 6144, 8)])   # the last two: rows above 48 KB
 def test_rotate_quantize_dual(P, orc, M, K, a_bits):
     spec = _spec(M, K, a_bits=a_bits)
     _codes_against_oracle(P, orc, spec, spec.activations(), f"dual {M}x{K}")
