@@ -559,7 +559,12 @@ def run_kernel(args):
     grid = default_clip_grid()
     stream = torch.cuda.current_stream()
     Wd = torch.from_numpy(s.weights()).to(dev)
-    tl = P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid)
+    # as in the whole-step workload: 3-bit codes of a small batch are stored packed and take the small-tile kernel
+    packed = s.w_bits == 3 and M <= 512
+    tl = P.lrq_tlq_quantize_weights(Wd, s.w_bits, s.group, 7, grid, grid,
+                                    code_layout=P.CODES_PACKED3 if packed else P.CODES_NIBBLE)
+    if packed:
+        args.gemm_impl = 2
     R = None if s.rot != "dense" else torch.from_numpy(s.rotation_bf16().view(np.int16)).view(torch.bfloat16).to(dev)
     kind = P.ROT_DENSE if s.rot == "dense" else P.ROT_HADAMARD
     L = P.QLayer(tl, s.N, s.K, kind, s.a_bits, s.had_block, R)
