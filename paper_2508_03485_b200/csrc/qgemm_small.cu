@@ -157,6 +157,20 @@ qgemm_small_kernel(const Params p) {
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     lrq_pdl_trigger();
+    if (threadIdx.x == 32) {
+        // The tile's weight codes and level tables do not depend on the previous kernel: ask for them in L2 now, while
+        // that kernel is still running, so that the main loop's first fetches do not start from DRAM.
+        const size_t w_pitch = PACKED3 ? (size_t)p.K * 3 / 8 : (size_t)p.K / 2;
+        const int rows = min(BN, p.N - n0);
+        const uint8_t* wc0 = p.w_codes + (size_t)n0 * w_pitch;
+        const size_t wbytes = (size_t)rows * w_pitch;
+        if (((reinterpret_cast<uintptr_t>(wc0) | wbytes) & 15) == 0)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(wc0), "r"((uint32_t)wbytes) : "memory");
+        const float* lv0 = p.levels + (size_t)n0 * (p.K / p.G) * NLEV;
+        const size_t lbytes = (size_t)rows * (p.K / p.G) * NLEV * sizeof(float);
+        if (((reinterpret_cast<uintptr_t>(lv0) | lbytes) & 15) == 0)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" :: "l"(lv0), "r"((uint32_t)lbytes) : "memory");
+    }
     lrq_pdl_wait();                      // the activation codes are the previous kernel's output
 
     if (warp < WORKERS / 32) {
