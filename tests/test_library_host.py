@@ -68,6 +68,18 @@ def test_argument_checks_run_before_any_launch(lib):
     assert lib.lrq_rotate_weights(fake, 8, 128, 128, None, 2, 0, None, fake, 128, None) == 1
     assert lib.lrq_rotate_weights(fake, 8, 128, 128, None, 2, 0, fake, fake, 128, None) == 1
     assert lib.lrq_rotate_weights(fake, 8, 128, 64, None, 0, 0, None, fake, 128, None) == 1      # ldw < K
+    # dual transformation: all three factors, blocks of 128, K a multiple of 128, scratch of 10 bytes per element
+    d = _ActParams(3, 0, None, 8, 0, None, 128, 0x1000, 0x1000, 0x1000)
+    assert lib.lrq_act_workspace_bytes(5, 256, C.byref(d)) == 5120 + 7680
+    assert lib.lrq_rotate_quantize_act(fake, 4, 256, 256, C.byref(d), fake, fake, fake, None, 0, None) == 3
+    assert lib.lrq_rotate_quantize_act(fake, 4, 192, 192, C.byref(d), fake, fake, fake, fake, 1 << 20, None) == 2
+    d_missing = _ActParams(3, 0, None, 8, 0, None, 128, 0x1000, None, 0x1000)
+    assert lib.lrq_rotate_quantize_act(fake, 4, 256, 256, C.byref(d_missing), fake, fake, fake, fake, 1 << 20, None) == 1
+    d64 = _ActParams(3, 0, None, 8, 0, None, 64, 0x1000, 0x1000, 0x1000)
+    assert lib.lrq_rotate_quantize_act(fake, 4, 256, 256, C.byref(d64), fake, fake, fake, fake, 1 << 20, None) == 2
+    assert lib.lrq_rotate_weights_dual(fake, 8, 256, 256, None, 128, fake, None, fake, fake, 256, None) == 1
+    assert lib.lrq_rotate_weights_dual(fake, 8, 200, 200, None, 128, fake, fake, fake, fake, 200, None) == 1
+    assert lib.lrq_static_scratch_bytes() == 8 << 20
     # rotation choice: 8 bytes of workspace, K a multiple of 16
     assert lib.lrq_ars_select(fake, 4, 128, 128, 1.0, fake, fake, None, 0, None) == 3
     assert lib.lrq_ars_select(fake, 4, 120, 120, 1.0, fake, fake, fake, 8, None) == 2
