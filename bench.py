@@ -432,10 +432,11 @@ def run_cuda(args):
 
     # A large batch goes through in token chunks (tokens are independent through the whole path): chunk c's outputs
     # travel back to the host while chunk c + 1 is computed, and its activations arrive while chunk c - 1 is computed.
-    # The chunks shrink towards the end: only the last chunk's read-back is left over when the kernels are done.
+    # The first and the last chunk are small: the kernels wait for the first chunk's upload only, and only the last
+    # chunk's read-back is left over when they are done.
     m_all = Xs[0].shape[0]
     chunked = m_all >= 16384 and m_all % 16 == 0 and all(x.shape[0] == m_all for x in Xs)
-    bounds = [0, m_all * 6 // 16, m_all * 11 // 16, m_all * 14 // 16, m_all] if chunked else [0, m_all]
+    bounds = [m_all * f // 16 for f in (0, 2, 7, 12, 15, 16)] if chunked else [0, m_all]
     nch = len(bounds) - 1
 
     def e2e_step():
