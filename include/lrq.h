@@ -248,7 +248,9 @@ lrq_status lrq_qlinear_stack(const lrq_layer* const* layers, int n_layers,
  * lrq_rotate_quantize_act.  `impl`: 0 = large-tile tcgen05 kernel (pairs of CTAs, 256 x 256 tiles), 1 = plain
  * CUDA-core kernel (kept as the in-library ablation baseline), 2 = small-tile tcgen05 kernel (128 x 32 tiles: the
  * one lrq_qlinear picks for a few hundred tokens or fewer, and the only tensor-core kernel that reads
- * LRQ_CODES_PACKED3).  LRQ_ERR_UNSUPPORTED when the kernel asked for does not take the layer's shape.
+ * LRQ_CODES_PACKED3), 3 = the integer form of Eq. 10 on the CUDA cores (mantissa products shifted by the level
+ * exponents, exact integer accumulation; I = 7 tables; a slow cross-check of the two forms, not a production path).
+ * LRQ_ERR_UNSUPPORTED when the kernel asked for does not take the layer's shape.
  * No workspace needed. */
 lrq_status lrq_qgemm_codes(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                            const int32_t* a_zp, int M, void* Y, lrq_dtype y_dtype, long ldy,

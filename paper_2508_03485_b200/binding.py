@@ -388,7 +388,8 @@ def lrq_qlinear_stack(plan: StackPlan, workspace: Optional[torch.Tensor] = None,
 def lrq_qgemm_codes(layer: QLayer, a_codes: torch.Tensor, a_scale: torch.Tensor, a_zp: torch.Tensor,
                     y_dtype: int = F32, impl: int = 0, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """Contraction + epilogue alone (Eq. 10) on codes from lrq_rotate_quantize_act.
-    impl 0: tcgen05 kernel, 1: CUDA-core baseline kernel."""
+    impl 0: large-tile tcgen05 kernel, 1: CUDA-core baseline, 2: small-tile tcgen05 kernel (the only tensor-core kernel for
+    packed 3-bit codes), 3: the integer shift form of Eq. 10 on the CUDA cores (exact sums; a slow cross-check)."""
     _need_cuda(a_codes, a_scale, a_zp, out)
     M = a_codes.shape[0]
     if out is None:

@@ -233,7 +233,8 @@ static lrq_status check_out(const void* Y, lrq_dtype dt, long ldy, int N) {
     return LRQ_OK;
 }
 
-// Which contraction kernel a call takes.  impl: 0 large-tile tcgen05, 1 CUDA cores, 2 small-tile tcgen05, -1 automatic:
+// Which contraction kernel a call takes.  impl: 0 large-tile tcgen05, 1 CUDA cores, 2 small-tile tcgen05, 3 CUDA cores
+// in the integer shift form, -1 automatic:
 // the small-tile kernel for packed 3-bit codes and for batches that give the large-tile kernel fewer tiles than half
 // the CTA pairs of the device (a few hundred tokens), the large-tile kernel otherwise, the CUDA cores for shapes
 // neither takes.
@@ -242,6 +243,7 @@ static lrq_status qgemm_dispatch(const lrq_layer* L, const uint8_t* a_codes, con
                                  cudaStream_t st) {
     if (impl == 1) return lrq_launch_qgemm_simple(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, st);
     if (impl == 2) return lrq_launch_qgemm_small(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, st);
+    if (impl == 3) return lrq_launch_qgemm_shift(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, st);
     if (impl == 0) return lrq_launch_qgemm_tc(L, a_codes, a_scale, a_zp, M, Y, dt, ldy, st);
     lrq_status s = LRQ_ERR_UNSUPPORTED;
     if (lrq_qgemm_small_takes(L)) {
@@ -259,7 +261,7 @@ extern "C" lrq_status lrq_qgemm_codes(const lrq_layer* L, const uint8_t* a_codes
                                       const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, int impl,
                                       void* cuda_stream) {
     if (!L || !a_codes || !a_scale || !a_zp || M <= 0) return LRQ_ERR_INVALID_ARG;
-    if (impl < 0 || impl > 2) return LRQ_ERR_INVALID_ARG;
+    if (impl < 0 || impl > 3) return LRQ_ERR_INVALID_ARG;
     lrq_status st = check_out(Y, dt, ldy, L->N);
     if (st != LRQ_OK) return st;
     if (!lrq_aligned(a_codes, 16)) return LRQ_ERR_INVALID_ARG;

@@ -104,6 +104,9 @@ __device__ __forceinline__ float lrq_ordered_float(int i) { return __int_as_floa
 // qgemm_simple.cu / qgemm_tc.cu
 lrq_status lrq_launch_qgemm_simple(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                                    const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);
+// qgemm_simple.cu : the integer form of Eq. 10 (mantissa products, shifts, exact integer accumulation) on the CUDA cores
+lrq_status lrq_launch_qgemm_shift(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
+                                  const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);
 lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const float* a_scale,
                                const int32_t* a_zp, int M, void* Y, lrq_dtype dt, long ldy, cudaStream_t st);
 // qgemm_small.cu : 128 x 32 tiles, one CTA each, for small token counts and for packed 3-bit codes
