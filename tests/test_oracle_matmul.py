@@ -108,3 +108,29 @@ def test_layer_rotation_invariance_with_fine_quantizers(orc):
     Y, *_ = orc.qlinear(X, T, 12, "hadamard", 64)
     ref = X @ W.T
     assert np.linalg.norm(Y - ref) / np.linalg.norm(ref) < 0.05
+
+
+def test_integer_shift_form_of_eq10_equals_the_level_table_product(orc):
+    # Eq. 10 as printed: (mantissa of the level x integer of the activation) << (f - I), with Python integers.  A level
+    # is II * 2^(f - I), II = rint(2^r * 2^I) (Eqs. 8-9, I = 7), so II and f come back exactly from the level's value.
+    import math
+    for G in (0, 8):
+        W, X, T, Q, S, Z = _tiny(orc, G=G, seed=10 + G)
+        Y = orc.qmatmul(Q, S, Z, T)
+        half, Gs = 4, (G or W.shape[1])
+        for n in range(W.shape[0]):
+            lv = T.levels[n].ravel()
+            exps = [math.frexp(abs(v))[1] for v in lv if v != 0.0]
+            emin = min(exps)                                   # common factor: keeps every shift non-negative
+            for m in range(X.shape[0]):
+                acc = 0
+                for k in range(W.shape[1]):
+                    v = float(T.levels[n, k // Gs, int(T.codes[n, k]) + half])
+                    f, e = math.frexp(abs(v))
+                    mant = int(f * 256)
+                    assert mant == f * 256 and 128 <= mant <= 255          # an 8-bit mantissa
+                    ix = int(Q[m, k]) + int(Z[m])                           # the activation's integer: x = s (q + z)
+                    acc += (-1 if v < 0 else 1) * ((mant * ix) << (e - emin)) if ix >= 0 else \
+                           (-1 if v < 0 else 1) * -((mant * -ix) << (e - emin))
+                exact = Fraction(float(S[m])) * Fraction(acc) * Fraction(2) ** (emin - 8)
+                assert abs(Y[m, n] - float(exact)) <= 1e-14 * max(1e-30, abs(float(exact)))
