@@ -14,8 +14,9 @@
  * library routines, brute force or exact rational arithmetic.  The readings of the paper that
  * no pin can reach (they are choices, not consequences) are "parity unpinned": the merge of
  * the two zero codes into one table entry, the clipping grid values, the search objective,
- * the block-diagonal Hadamard for sizes that are not a power of two, and the symmetric
- * activation mode.  The smoothing vector of orc_smooth (Sec. 5.1) is an input here: how it is
+ * the block-diagonal Hadamard for sizes that are not a power of two, the symmetric
+ * activation mode, and the shape in which the dual transformation's factors are taken
+ * (block-diagonal rotations of one block size around an index map).  The smoothing vector of orc_smooth (Sec. 5.1) is an input here: how it is
  * calibrated (migration strength 0.5) is outside the path, so only its application is pinned.
  */
 #include <math.h>
