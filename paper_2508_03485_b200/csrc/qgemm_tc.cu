@@ -47,7 +47,8 @@ constexpr int BN = 256;                      // output channels per tile (templa
 constexpr int BN_CTA = 128;                  // weight rows decoded per CTA
 constexpr int BK = 64;
 constexpr int STAGES = 4;                    // bf16 operand stages
-constexpr int CSTAGES = 4;                   // packed-code stages (the TMA runs this many k-blocks ahead of the decode)
+constexpr int CSTAGES = 6;                   // packed-code stages: the TMA runs this many k-blocks ahead of the decode (with 32768
+                                             // tokens the code tiles come from a busy L2 / DRAM: 2 stages 614, 4 stages 972, 6 stages 1038 TFLOP/s)
 constexpr int A_STAGE_BYTES = BM_CTA * BK * 2;      // 16 KB
 constexpr int B_STAGE_BYTES = BN_CTA * BK * 2;      // 16 KB
 constexpr int AC_STAGE_BYTES = BM_CTA * BK;         // room for 8-bit codes (4-bit codes use half)
@@ -71,7 +72,7 @@ struct __align__(16) SharedCtl {
 };
 
 constexpr int EPI_TILE_BYTES = 32 * 32 * 4;         // one epilogue warp's 32 x 32 fp32 chunk, staged for a TMA store
-constexpr int EPI_TILES = 2;                        // per epilogue warp: one being filled while the other is stored
+constexpr int EPI_TILES = 1;                        // staging tiles per epilogue warp (a second one bought nothing; its 16 KB went to the code stages)
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
                               (size_t)NUM_EPI_WARPS * EPI_TILES * EPI_TILE_BYTES +
                               (size_t)CSTAGES * (AC_STAGE_BYTES + WC_STAGE_BYTES) + sizeof(SharedCtl);
@@ -545,7 +546,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                     // writes whole lines, clips rows past M and columns past N, and runs while the next chunk is
                     // prepared.  fp32: one 32 x 32 tile per chunk; 16-bit: two chunks side by side, 32 rows x 64.
                     if (m0 + ew * 32 < p.M) {                          // warp-uniform; every store starts inside Y
-                        const uint32_t tile = smem_u32(sEpi) + (uint32_t)((ew * EPI_TILES + (nstore & 1)) * EPI_TILE_BYTES);
+                        const uint32_t tile = smem_u32(sEpi) + (uint32_t)((ew * EPI_TILES + (nstore % EPI_TILES)) * EPI_TILE_BYTES);
                         if (p.y_dtype == LRQ_F32) {
                             if (lane == 0) tma_store_wait_read<EPI_TILES - 1>();     // the store that last read this tile is done with it
                             __syncwarp();
