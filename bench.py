@@ -41,7 +41,7 @@ from lrq_workloads import bf16_bits_to_f64, config_layers, default_clip_grid  # 
 # kernel changes after the capture.
 NCU_TRAFFIC_BYTES = {
     "qgemm cfg4 b0.fc1": 65.20e6 + 547.50e6,
-    "qgemm cfg3 fc1": None,
+    "qgemm cfg3 fc1": 27.10e6 + 169.40e6,
     "rotq cfg4 b0.fc2": 303.10e6 + 117.94e6,
     "rotq cfg3 fc2": 113.27e6 + 11.70e6,
     "rotgemm cfg3 qkv": 51.51e6 + 19.17e6 + 56.67e6 + 0.25e6,
@@ -49,7 +49,7 @@ NCU_TRAFFIC_BYTES = {
 
 # sm__pipe_tensor_cycles_active (% of elapsed cycles) of the same captures: the tensor pipe's own view of the
 # contraction, beside the fraction of the measured matmul peak that `frac` reports
-NCU_TENSOR_PIPE_PCT = {"qgemm cfg4 b0.fc1": 48.4, "qgemm cfg3 fc1": 53.8}
+NCU_TENSOR_PIPE_PCT = {"qgemm cfg4 b0.fc1": 48.4, "qgemm cfg3 fc1": 54.2}
 
 METRIC = "qlinear_tflops"
 UNIT = "TFLOP/s"

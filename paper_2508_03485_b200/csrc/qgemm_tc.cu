@@ -217,7 +217,7 @@ using namespace lrq_f2;
 struct Params {
     const float* a_scale; const int32_t* a_zp;
     const float* levels; const float* wsum; const float* wscale; const float* bias;
-    void* Y; long ldy; int M, N, K, G, y_dtype; int* status;
+    void* Y; long ldy; int M, N, K, G, y_dtype; int col_fastest; int* status;
 };
 
 template <int A_BITS, int W_BITS, int BN_T>
@@ -240,9 +240,17 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
     constexpr uint32_t IDESC = umma_idesc_bf16(2 * BM_CTA, BN_T, false, false);
     const int tiles_m = (p.M + 2 * BM_CTA - 1) / (2 * BM_CTA), tiles_n = (p.N + BN_T - 1) / BN_T;
     const int num_tiles = tiles_m * tiles_n;
-    // a pair takes a contiguous run of tiles in the order (token tile, column tile) with the column fastest: its
-    // consecutive tiles share their activation codes, which then come from DRAM once
-    const int tile_first = (int)(((long long)pair * num_tiles) / num_pairs), tile_last = (int)(((long long)(pair + 1) * num_tiles) / num_pairs);
+    // Which tiles a pair takes, and in which order.  col_fastest (the activation codes outweigh the weight codes: many
+    // tokens): a contiguous run of tiles in the order (token tile, column tile) with the column fastest, so that the
+    // pair's consecutive tiles share their activation codes, which then come from DRAM once.  Otherwise (few tokens, a
+    // large weight matrix): round-robin with the token tile fastest, so that the pairs running at the same time share
+    // a tile column's weight codes.
+    const bool col_fastest = p.col_fastest != 0;
+    const int tile_first = col_fastest ? (int)(((long long)pair * num_tiles) / num_pairs) : pair;
+    const int tile_last = col_fastest ? (int)(((long long)(pair + 1) * num_tiles) / num_pairs) : num_tiles;
+    const int tile_step = col_fastest ? 1 : num_pairs;
+    auto tile_m = [&](int t) { return col_fastest ? t / tiles_n : t % tiles_m; };
+    auto tile_n = [&](int t) { return col_fastest ? t % tiles_n : t / tiles_m; };
     const int kblocks = p.K / BK;
     constexpr int NLEV = 1 << W_BITS;
     constexpr int AC_ROW_BYTES = BK * A_BITS / 8;                   // 64 or 32 code bytes per token and k-block
@@ -283,9 +291,9 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = tile_first; tile < tile_last && ok; ++tile) {
-                const int m_base = (tile / tiles_n) * 2 * BM_CTA + (int)rank * BM_CTA;
-                const int n_base = (tile % tiles_n) * BN_T + (int)rank * BN_CTA_T;
+            for (int tile = tile_first; tile < tile_last && ok; tile += tile_step) {
+                const int m_base = tile_m(tile) * 2 * BM_CTA + (int)rank * BM_CTA;
+                const int n_base = tile_n(tile) * BN_T + (int)rank * BN_CTA_T;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int cs = it % CSTAGES;
                     ok = mbar_wait<200>(smem_u32(&ctl->cempty[cs]), ((it / CSTAGES) & 1) ^ 1, &ctl->abort_flag, p.status, 1);
@@ -311,7 +319,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         if (rank == 0 && lane == 0) {
             uint32_t it = 0, t = 0;
             bool ok = true;
-            for (int tile = tile_first; tile < tile_last && ok; ++tile, ++t) {
+            for (int tile = tile_first; tile < tile_last && ok; tile += tile_step, ++t) {
                 const int buf = t & 1;
                 ok = mbar_wait_cluster<64>(smem_u32(&ctl->tmem_empty[buf]), ((t >> 1) & 1) ^ 1, &ctl->abort_flag, p.status, 4);
                 if (!ok) break;
@@ -353,8 +361,8 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         uint32_t it0 = 0;
         bool ok = true, have_next = false;
         float4 raw[NLEV / 4];
-        for (int tile = tile_first; tile < tile_last && ok; ++tile, it0 += kblocks) {
-            const int n_base = (tile % tiles_n) * BN_T + (int)rank * BN_CTA_T;
+        for (int tile = tile_first; tile < tile_last && ok; tile += tile_step, it0 += kblocks) {
+            const int n_base = tile_n(tile) * BN_T + (int)rank * BN_CTA_T;
             const int n = min(n_base + row, p.N - 1);               // rows past N decode a valid table; never stored
             const float4* tab = reinterpret_cast<const float4*>(p.levels + (size_t)n * ngrp * NLEV);
             const int kb0 = (grp ^ (int)it0) & 1;
@@ -369,9 +377,9 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
                 build_lut<W_BITS>(L, raw);
             }
             have_next = false;
-            if (ngrp == 1 && tile + 1 < tile_last) {
+            if (ngrp == 1 && tile + tile_step < tile_last) {
                 // per-channel tables: the next tile's table is fetched now, a whole tile before it is needed
-                const int nn = min(((tile + 1) % tiles_n) * BN_T + (int)rank * BN_CTA_T + row, p.N - 1);
+                const int nn = min(tile_n(tile + tile_step) * BN_T + (int)rank * BN_CTA_T + row, p.N - 1);
                 const float4* tn = reinterpret_cast<const float4*>(p.levels + (size_t)nn * NLEV);
 #pragma unroll
                 for (int j = 0; j < NLEV / 4; ++j) raw[j] = __ldg(tn + j);
@@ -447,7 +455,7 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         RingPos ring(grp);
         uint32_t it0 = 0;
         bool ok = true;
-        for (int tile = tile_first; tile < tile_last && ok; ++tile, it0 += kblocks) {
+        for (int tile = tile_first; tile < tile_last && ok; tile += tile_step, it0 += kblocks) {
             for (int kb = (grp ^ (int)it0) & 1; kb < kblocks; kb += 2) {
                 ok = mbar_wait_warp<64>(smem_u32(&ctl->cfull[ring.cs]), ring.cph, &ctl->abort_flag, p.status, 6);
                 if (!ok) break;
@@ -492,8 +500,8 @@ qgemm_tc_kernel(const Params p, const __grid_constant__ CUtensorMap tmA, const _
         const float zoff = (A_BITS == 8) ? 128.f : 8.f;            // the A operand is fed as q - 128 / q - 8
         const bool has_ws = p.wscale != nullptr, has_bias = p.bias != nullptr;
         uint32_t t = 0, nstore = 0;
-        for (int tile = tile_first; tile < tile_last; ++tile, ++t) {
-            const int m0 = (tile / tiles_n) * 2 * BM_CTA + (int)rank * BM_CTA, n0 = (tile % tiles_n) * BN_T;
+        for (int tile = tile_first; tile < tile_last; tile += tile_step, ++t) {
+            const int m0 = tile_m(tile) * 2 * BM_CTA + (int)rank * BM_CTA, n0 = tile_n(tile) * BN_T;
             const int buf = t & 1;
             // stage the tile's per-column terms (wsum, wscale, bias) in shared memory
             float (*col)[BN] = ctl->col[buf];
@@ -695,6 +703,8 @@ lrq_status lrq_launch_qgemm_tc(const lrq_layer* L, const uint8_t* a_codes, const
     p.a_scale = a_scale; p.a_zp = a_zp;
     p.levels = L->levels; p.wsum = L->wsum; p.wscale = L->wscale; p.bias = L->bias;
     p.Y = Y; p.ldy = ldy; p.M = M; p.N = L->N; p.K = L->K; p.G = L->group; p.y_dtype = (int)dt;
+    // tile order: the operand whose codes weigh more is the one a pair keeps while it walks the other
+    p.col_fastest = (size_t)M * ab > (size_t)L->N * 4 ? 1 : 0;      // M*K*ab/8 bytes of activation codes against N*K/2
     p.status = lrq_status_word();
     int sms = 0;
     if (lrq_current_device(nullptr, &sms) != LRQ_OK) return LRQ_ERR_CUDA;
